@@ -1,0 +1,204 @@
+/*
+ * palsgd.h -- C ABI of the PALSGD update / synchronisation library (CUDA, sm_100a).
+ *
+ * The library runs the per-step parameter arithmetic of Pseudo-Asynchronous
+ * Local SGD (Algorithm 1 of the paper) for K data-parallel workers that live as
+ * K replica slots in ONE GPU's memory:
+ *
+ *   - the inner optimizer step of every worker (AdamW or momentum SGD) with the
+ *     rescaled step size alpha_t / (1 - p)                    [Algorithm 1; Eq. (1)]
+ *   - the probabilistic pseudo-synchronisation that pulls a worker's local model
+ *     x_k toward its copy x of the global model with coefficient
+ *     alpha_t * eta_t / p                                     [Algorithm 1; Eq. (2)]
+ *   - every H steps the outer synchronisation: average of the K local models
+ *     (Sec. 2.2), outer gradient Delta = x - average (Eq. (3)), OuterOPT = SGD
+ *     with (Nesterov) momentum (Eq. (4); Sec. 4.3), and the restart of every
+ *     worker from the new global model (Sec. 3.1).
+ *
+ * General rules
+ *   - Every entry point returns a palsgd_status (0 = PALSGD_OK, negative = error),
+ *     never throws, never exits.  palsgd_strerror() names a status.
+ *   - All parameter/gradient/state buffers are DEVICE memory owned by the caller;
+ *     they must stay valid until palsgd_destroy().  The library allocates only
+ *     its context and a few KB..MB of device tables (chunk table, pointer
+ *     tables, a counter block); palsgd_destroy() frees them.
+ *   - `stream` arguments are a cudaStream_t passed as void* (NULL = the legacy
+ *     default stream).  Work is enqueued asynchronously unless stated otherwise.
+ *     Successive calls on one context must be stream-ordered with each other.
+ *   - A context is not thread-safe; distinct contexts are independent.
+ *   - Buffers need only natural element alignment.  Tensors whose every buffer
+ *     is 16-byte aligned take the 128-bit vector path; others a scalar path
+ *     with identical results.
+ *   - Arithmetic: every element operation is one IEEE binary32 operation in the
+ *     order documented at each call (no fused multiply-add, round-to-nearest
+ *     division and square root).  Scalars (step sizes, bias corrections) are
+ *     formed in binary64 and rounded once.
+ */
+#ifndef PALSGD_H_
+#define PALSGD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define PALSGD_MAX_WORKERS 64u
+
+typedef struct palsgd_ctx palsgd_ctx;   /* opaque; created by palsgd_init, freed by palsgd_destroy */
+
+typedef enum palsgd_status {
+    PALSGD_OK           =  0,
+    PALSGD_EINVAL       = -1,   /* NULL pointer, K = 0 or > 64, H = 0, p outside [0,1], bad enum ... */
+    PALSGD_EALIGN       = -2,   /* a pointer is not aligned to its element size                      */
+    PALSGD_ECUDA        = -3,   /* a CUDA runtime call or a kernel launch failed                     */
+    PALSGD_ESTATE       = -4,   /* call not valid in this state (e.g. undefined coefficient)         */
+    PALSGD_ENOMEM       = -5,   /* host or device allocation failed                                  */
+    PALSGD_EUNSUPPORTED = -6    /* combination not built                                             */
+} palsgd_status;
+
+enum { PALSGD_INNER_ADAMW = 0, PALSGD_INNER_SGDM = 1 };
+enum { PALSGD_PREC_FP32 = 0, PALSGD_PREC_BF16_MASTER = 1 };
+
+/* Algorithm 1's data line: K, p, H, InnerOPT, OuterOPT.  (alpha_t and eta_t are
+ * per-call arguments because the paper indexes them by t.) */
+typedef struct palsgd_config {
+    uint32_t K;               /* number of workers / replica slots, 1..64                        */
+    int32_t  inner;           /* PALSGD_INNER_ADAMW | PALSGD_INNER_SGDM                          */
+    uint64_t H;               /* outer-sync interval, >= 1                                       */
+    double   p;               /* probability of the pseudo-sync branch, in [0, 1]                */
+    double   beta1, beta2;    /* AdamW moment decay rates                                        */
+    double   eps;             /* AdamW epsilon (added to sqrt of the corrected second moment)    */
+    double   weight_decay;    /* AdamW: decoupled; SGD: L2 term added to the gradient            */
+    double   momentum;        /* inner SGD momentum (ignored by AdamW)                           */
+    double   outer_lr;        /* OuterOPT learning rate                                          */
+    double   outer_momentum;  /* OuterOPT momentum; (outer_lr, outer_momentum, nesterov) =       */
+    int32_t  outer_nesterov;  /*   (1, 0, 0) is plain averaging (Local SGD / Theorem 1)          */
+    int32_t  precision;       /* PALSGD_PREC_FP32 | PALSGD_PREC_BF16_MASTER                      */
+    uint64_t seed;            /* seed of the decision stream                                     */
+} palsgd_config;
+
+/* Caller-owned device buffers.  Arrays of K*n_tensors pointers are indexed
+ * [k * n_tensors + j] (worker k, tensor j); arrays of n_tensors pointers by [j].
+ * The pointer ARRAYS themselves are host memory and are copied by palsgd_init. */
+typedef struct palsgd_buffers {
+    void* const*       param;      /* [K*n] local models x_k: float (FP32) or bfloat16 working
+                                      copy (BF16_MASTER; overwritten by init with RNE(master))   */
+    const void* const* grad;       /* [K*n] gradients g_k: float (FP32) or bfloat16; read only   */
+    float* const*      master;     /* [K*n] fp32 master of x_k (BF16_MASTER) else NULL           */
+    float* const*      m;          /* [K*n] AdamW first moment / SGD momentum buffer             */
+    float* const*      v;          /* [K*n] AdamW second moment; NULL for SGD                    */
+    float* const*      global;     /* [n]   global model copy x (written by init)                */
+    float* const*      outer_mom;  /* [n]   OuterOPT momentum buffer u (zeroed by init)          */
+} palsgd_buffers;
+
+/*
+ * Create a context (Algorithm 1, initialisation).  Validates everything before
+ * touching the GPU.  Then, on `stream`: m, v, outer_mom <- 0; global[i] <-
+ * (x_0[i] + x_1[i] + ... + x_{K-1}[i]) / K, summed in that order (Sec. 2.2; the
+ * paper starts all workers from one x^(0), for which this is x^(0)); in
+ * BF16_MASTER mode param <- RNE_bf16(master).  Counters t, s_k, n_outer <- 0.
+ * numel[j] is the element count of tensor j (0 allowed).  Tensors that are
+ * adjacent in memory in every buffer are fused into one segment internally.
+ * Errors: EINVAL / EALIGN before any CUDA call; ENOMEM; ECUDA.
+ */
+int palsgd_init(palsgd_ctx** out, const palsgd_config* cfg, size_t n_tensors,
+                const uint64_t* numel, const palsgd_buffers* bufs, void* stream);
+
+/*
+ * One pass of Algorithm 1's inner loop body for all K workers, ONE kernel launch.
+ * For worker k the kernel draws b_k^(t) ("b ~ U[0,1]; b <= p"): the first word r of
+ * Philox4x32-10 with key (seed_lo, seed_hi) and counter (t_lo, t_hi, k, 0);
+ * b = (r < floor(p * 2^32)).  One draw per (worker, step) for the whole model.
+ *   b = 1, Eq. (2):  d = x - x_g;  x = x - beta * d,   beta = fl32(alpha_t*eta_t/p).
+ *          Gradient, moments and s_k are not touched.
+ *   b = 0, Eq. (1):  s_k += 1;  lr = fl32(alpha_t/(1-p)) and
+ *     AdamW:  m = b1*m + (1-b1)*g;  v = b2*v + (1-b2)*(g*g);
+ *             mh = m / (1-b1^s_k);  vh = v / (1-b2^s_k);
+ *             x = x * fl32(1 - lr*wd);  x = x - lr * (mh / (sqrt(vh) + eps))
+ *     SGD:    g' = g + wd*x;  m = mu*m + g';  x = x - lr*m
+ * In BF16_MASTER mode x above is the fp32 master, g is widened exactly, and the
+ * bf16 working copy is rewritten as RNE(master).  Afterwards t += 1 (device side).
+ * Does NOT run the outer sync; see palsgd_step.
+ * Errors: EINVAL (NULL ctx, non-finite or negative rates); ECUDA.
+ */
+int palsgd_inner_step(palsgd_ctx* ctx, double lr_t, double eta_t, void* stream);
+
+/*
+ * A pull imposed on the workers whose bit is set in worker_mask, with the mixing
+ * coefficient given directly (the EMA form after Eq. (2): x_k <- (1-beta) x_k +
+ * beta x, computed as x - beta*(x - x_g)).  No draw; t, s_k unchanged.
+ * Errors: EINVAL (NULL ctx, mask bit >= K, non-finite beta); ECUDA.
+ */
+int palsgd_pseudo_sync(palsgd_ctx* ctx, uint64_t worker_mask, double beta, void* stream);
+
+/*
+ * Outer synchronisation, ONE kernel launch (Algorithm 1, "(t+1) mod H = 0" block):
+ *   xbar = (x_0 + x_1 + ... + x_{K-1}) / K      (that order; Sec. 2.2)
+ *   Delta = x_g - xbar                          (Eq. (3))
+ *   u = mu*u + Delta;  x_g = x_g - lr_out*(Delta + mu*u)   (Nesterov; Eq. (4))
+ *                      x_g = x_g - lr_out*u                (outer_nesterov = 0)
+ *   x_k = x_g for every k  (Sec. 3.1: every worker restarts from the global model)
+ * Inner optimizer state is kept.  n_outer += 1.  BF16_MASTER: masters are
+ * averaged; masters and bf16 working copies are rewritten.
+ * Errors: EINVAL (NULL ctx); ECUDA.
+ */
+int palsgd_outer_sync(palsgd_ctx* ctx, void* stream);
+
+/* Algorithm 1, one iteration t: palsgd_inner_step, then palsgd_outer_sync when
+ * the number of completed steps is a multiple of H. */
+int palsgd_step(palsgd_ctx* ctx, double lr_t, double eta_t, void* stream);
+
+/*
+ * palsgd_step with HOST gradients and HOST results (the end-to-end call):
+ * copies h_grad[k*n_tensors+j] (host, numel[j] elements of the gradient type;
+ * pinned memory makes the copies asynchronous) into the gradient buffers, runs
+ * palsgd_step, copies the K decisions of this step to h_decisions (K bytes, may
+ * be NULL) and, if this step ended with an outer sync and h_global is not NULL,
+ * the new global model to h_global[j] (float, numel[j] each).  *synced (may be
+ * NULL) receives 1 if the outer sync ran.  SYNCHRONISES the stream before
+ * returning.  Errors: as palsgd_step.
+ */
+int palsgd_step_host(palsgd_ctx* ctx, const void* const* h_grad, double lr_t, double eta_t,
+                     float* const* h_global, uint8_t* h_decisions, int* synced, void* stream);
+
+/*
+ * Read the counters (SYNCHRONISES the stream): t = completed steps, s_k[K] =
+ * gradient steps taken by worker k, n_outer = outer syncs, last_b[K] = decisions
+ * of the latest inner step.  Any output pointer may be NULL.
+ * Errors: ESTATE if the device-side t disagrees with the host mirror; ECUDA.
+ */
+int palsgd_get_counters(palsgd_ctx* ctx, uint64_t* t, uint64_t* s_k, uint64_t* n_outer,
+                        uint8_t* last_b, void* stream);
+
+/* Resume: set t, s_k[K], n_outer (the decision stream is a pure function of
+ * (seed, t, k), so a restored run continues bit-exactly).  Enqueued on stream. */
+int palsgd_set_counters(palsgd_ctx* ctx, uint64_t t, const uint64_t* s_k, uint64_t n_outer,
+                        void* stream);
+
+/* Number of kernels this context has launched so far (host-side count). */
+int palsgd_get_launch_count(palsgd_ctx* ctx, uint64_t* n_launches);
+
+/* Launch-shape knobs (advanced; results never depend on them).  value = the
+ * largest grid a launch may use, CTAs looping over work items beyond it;
+ * 0 (default) = one CTA per work item. */
+enum { PALSGD_TUNE_INNER_GRID_CAP = 0, PALSGD_TUNE_OUTER_GRID_CAP = 1 };
+int palsgd_set_tuning(palsgd_ctx* ctx, int knob, int64_t value);
+
+/* The branch draw as a pure host function: 1 = pseudo-sync, 0 = gradient step;
+ * negative status on bad arguments (p outside [0,1], k >= 64). */
+int palsgd_decision(uint64_t seed, uint64_t t, uint32_t k, double p);
+
+/* Text for a status; the CUDA error string of the latest ECUDA on ctx (or ""). */
+const char* palsgd_strerror(int status);
+const char* palsgd_last_cuda_error(palsgd_ctx* ctx);
+
+/* Free the context and its device tables.  NULL is accepted.  The caller's
+ * buffers are not touched. */
+void palsgd_destroy(palsgd_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PALSGD_H_ */

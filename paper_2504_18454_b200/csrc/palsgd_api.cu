@@ -1,0 +1,540 @@
+// Host controller and C ABI of the PALSGD library (see include/palsgd.h).
+//
+// The controller validates arguments, fuses adjacent tensors into segments,
+// builds the chunk table and pointer tables once, forms the per-call scalars
+// in binary64, and launches one kernel per call.  Counters that the kernels
+// need (t, s_k, beta^s_k) live on the device; the host keeps a mirror of t and
+// n_outer for the "(t+1) mod H" test.
+#include "../../include/palsgd.h"
+
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "palsgd_kernels.cuh"
+
+using namespace palsgd;
+
+struct Segment {
+    size_t   first_tensor;
+    size_t   n_tensors;
+    uint64_t numel;
+};
+
+struct palsgd_ctx {
+    palsgd_config cfg{};
+    size_t n_tensors = 0;
+    std::vector<uint64_t> numel;
+    std::vector<Segment> segs;
+    // host copies of the caller's pointer arrays (for the host-buffer entry point)
+    std::vector<const void*> h_grad_dev;     // [K*n_tensors] device gradient pointers
+    std::vector<float*> h_global_dev;        // [n_tensors]
+    // device tables
+    void* d_blob = nullptr;                  // one allocation holding everything below
+    Tables tb{};
+    uint64_t P = 0;
+    // host mirrors
+    uint64_t t = 0, n_outer = 0, launches = 0;
+    uint64_t thr = 0;
+    int grid_cap_inner = 0, grid_cap_outer = 0;   // 0 = one CTA per work item
+    std::string cuda_err;
+};
+
+namespace {
+
+thread_local std::string g_noctx_err;
+
+int cuda_fail(palsgd_ctx* ctx, cudaError_t e, const char* what)
+{
+    std::string msg = std::string(what) + ": " + cudaGetErrorString(e);
+    if (ctx) ctx->cuda_err = msg; else g_noctx_err = msg;
+    return PALSGD_ECUDA;
+}
+
+#define PALSGD_CUDA(ctx, call)                                            \
+    do { cudaError_t e_ = (call); if (e_ != cudaSuccess) return cuda_fail((ctx), e_, #call); } while (0)
+
+inline bool finite_nonneg(double v) { return std::isfinite(v) && v >= 0.0; }
+inline size_t elem_size_param(int prec) { return prec == PALSGD_PREC_BF16_MASTER ? 2 : 4; }
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+uint64_t threshold_of(double p) { return (uint64_t)std::floor(p * 4294967296.0); }
+
+int validate_config(const palsgd_config* c)
+{
+    if (!c) return PALSGD_EINVAL;
+    if (c->K == 0 || c->K > PALSGD_MAX_WORKERS) return PALSGD_EINVAL;
+    if (c->H == 0) return PALSGD_EINVAL;
+    if (!(c->p >= 0.0 && c->p <= 1.0)) return PALSGD_EINVAL;
+    if (c->inner != PALSGD_INNER_ADAMW && c->inner != PALSGD_INNER_SGDM) return PALSGD_EINVAL;
+    if (c->precision != PALSGD_PREC_FP32 && c->precision != PALSGD_PREC_BF16_MASTER) return PALSGD_EINVAL;
+    if (c->outer_nesterov != 0 && c->outer_nesterov != 1) return PALSGD_EINVAL;
+    if (c->inner == PALSGD_INNER_ADAMW) {
+        if (!(c->beta1 >= 0.0 && c->beta1 < 1.0) || !(c->beta2 >= 0.0 && c->beta2 < 1.0)) return PALSGD_EINVAL;
+        if (!finite_nonneg(c->eps)) return PALSGD_EINVAL;
+    } else {
+        if (!finite_nonneg(c->momentum)) return PALSGD_EINVAL;
+    }
+    if (!finite_nonneg(c->weight_decay)) return PALSGD_EINVAL;
+    if (!std::isfinite(c->outer_lr) || !finite_nonneg(c->outer_momentum)) return PALSGD_EINVAL;
+    return PALSGD_OK;
+}
+
+// Pointer of buffer kind `kind` for (k, j); kinds: 0 param 1 grad 2 master 3 m 4 v
+const void* buf_ptr(const palsgd_buffers* b, int kind, size_t idx)
+{
+    switch (kind) {
+        case 0: return b->param[idx];
+        case 1: return b->grad[idx];
+        case 2: return b->master[idx];
+        case 3: return b->m[idx];
+        default: return b->v[idx];
+    }
+}
+
+template <typename F>
+int launch_checked(palsgd_ctx* ctx, F&& launch)
+{
+    launch();
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "kernel launch");
+    ctx->launches += 1;
+    return PALSGD_OK;
+}
+
+unsigned grid_for(uint64_t n_items, int cap)
+{
+    uint64_t g = n_items;
+    if (cap > 0 && g > (uint64_t)cap) g = (uint64_t)cap;
+    if (g > 0x7FFFFFFFull) g = 0x7FFFFFFFull;
+    return (unsigned)(g == 0 ? 1 : g);
+}
+
+OuterArgs outer_args(const palsgd_ctx* ctx)
+{
+    OuterArgs a{};
+    a.tb = ctx->tb;
+    a.mu = (float)ctx->cfg.outer_momentum;
+    a.lr = (float)ctx->cfg.outer_lr;
+    a.Kf = (float)ctx->cfg.K;
+    a.nesterov = ctx->cfg.outer_nesterov;
+    return a;
+}
+
+int launch_inner(palsgd_ctx* ctx, const InnerArgs& a, cudaStream_t s)
+{
+    const uint64_t n_items = (uint64_t)ctx->tb.n_chunks * ctx->cfg.K;
+    // with nothing to stream a one-CTA launch still advances the counters
+    const unsigned grid = grid_for(n_items, ctx->grid_cap_inner);
+    const bool adam = ctx->cfg.inner == PALSGD_INNER_ADAMW;
+    const bool bf = ctx->cfg.precision == PALSGD_PREC_BF16_MASTER;
+    return launch_checked(ctx, [&] {
+        if (adam && !bf)      palsgd_inner_kernel<0, 0, 4><<<grid, kThreads, 0, s>>>(a);
+        else if (!adam && !bf) palsgd_inner_kernel<1, 0, 4><<<grid, kThreads, 0, s>>>(a);
+        else if (adam && bf)  palsgd_inner_kernel<0, 1, 2><<<grid, kThreads, 0, s>>>(a);
+        else                  palsgd_inner_kernel<1, 1, 2><<<grid, kThreads, 0, s>>>(a);
+    });
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------------- init
+
+extern "C" int palsgd_init(palsgd_ctx** out, const palsgd_config* cfg, size_t n_tensors,
+                           const uint64_t* numel, const palsgd_buffers* bufs, void* stream)
+{
+    if (!out) return PALSGD_EINVAL;
+    *out = nullptr;
+    int rc = validate_config(cfg);
+    if (rc) return rc;
+    if (n_tensors == 0 || !numel || !bufs) return PALSGD_EINVAL;
+    const uint32_t K = cfg->K;
+    const bool bf = cfg->precision == PALSGD_PREC_BF16_MASTER;
+    const bool adam = cfg->inner == PALSGD_INNER_ADAMW;
+    if (!bufs->param || !bufs->grad || !bufs->m || !bufs->global || !bufs->outer_mom) return PALSGD_EINVAL;
+    if (bf && !bufs->master) return PALSGD_EINVAL;
+    if (adam && !bufs->v) return PALSGD_EINVAL;
+
+    // which buffer kinds exist, and their element sizes
+    const size_t ps = elem_size_param(cfg->precision);
+    struct Kind { int id; size_t esize; bool present; };
+    const Kind kinds[5] = {{0, ps, true}, {1, ps, true}, {2, 4, bf}, {3, 4, true}, {4, 4, adam}};
+
+    uint64_t P = 0;
+    for (size_t j = 0; j < n_tensors; ++j) {
+        if (numel[j] > (1ull << 40)) return PALSGD_EINVAL;
+        P += numel[j];
+        for (uint32_t k = 0; k < K; ++k) {
+            const size_t idx = (size_t)k * n_tensors + j;
+            for (const Kind& kd : kinds) {
+                if (!kd.present) continue;
+                const void* p = buf_ptr(bufs, kd.id, idx);
+                if (!p && numel[j] > 0) return PALSGD_EINVAL;
+                if (!aligned(p, kd.esize)) return PALSGD_EALIGN;
+            }
+        }
+        if ((!bufs->global[j] || !bufs->outer_mom[j]) && numel[j] > 0) return PALSGD_EINVAL;
+        if (!aligned(bufs->global[j], 4) || !aligned(bufs->outer_mom[j], 4)) return PALSGD_EALIGN;
+    }
+
+    palsgd_ctx* ctx = new (std::nothrow) palsgd_ctx();
+    if (!ctx) return PALSGD_ENOMEM;
+    ctx->cfg = *cfg;
+    ctx->n_tensors = n_tensors;
+    ctx->numel.assign(numel, numel + n_tensors);
+    ctx->P = P;
+    ctx->thr = threshold_of(cfg->p);
+    ctx->h_grad_dev.assign(bufs->grad, bufs->grad + (size_t)K * n_tensors);
+    ctx->h_global_dev.assign(bufs->global, bufs->global + n_tensors);
+
+    // ---- fuse tensors that are adjacent in every buffer into segments
+    auto adjacent = [&](size_t j) {           // is tensor j+1 right behind tensor j everywhere?
+        for (uint32_t k = 0; k < K; ++k) {
+            const size_t a = (size_t)k * n_tensors + j, b = a + 1;
+            for (const Kind& kd : kinds) {
+                if (!kd.present) continue;
+                const char* pa = static_cast<const char*>(buf_ptr(bufs, kd.id, a));
+                const char* pb = static_cast<const char*>(buf_ptr(bufs, kd.id, b));
+                if (pa + numel[j] * kd.esize != pb) return false;
+            }
+        }
+        const char* ga = reinterpret_cast<const char*>(bufs->global[j]);
+        const char* ua = reinterpret_cast<const char*>(bufs->outer_mom[j]);
+        return ga + numel[j] * 4 == reinterpret_cast<const char*>(bufs->global[j + 1]) &&
+               ua + numel[j] * 4 == reinterpret_cast<const char*>(bufs->outer_mom[j + 1]);
+    };
+    for (size_t j = 0; j < n_tensors;) {
+        Segment sg{j, 1, numel[j]};
+        while (sg.first_tensor + sg.n_tensors < n_tensors &&
+               adjacent(sg.first_tensor + sg.n_tensors - 1)) {
+            sg.numel += numel[sg.first_tensor + sg.n_tensors];
+            sg.n_tensors += 1;
+        }
+        j += sg.n_tensors;
+        if (sg.numel > 0) ctx->segs.push_back(sg);
+    }
+    const size_t n_seg = ctx->segs.size();
+
+    // ---- chunk table and per-segment vector-path flag
+    std::vector<Chunk> chunks;
+    for (size_t s = 0; s < n_seg; ++s) {
+        const Segment& sg = ctx->segs[s];
+        bool vec = aligned(bufs->global[sg.first_tensor], 16) && aligned(bufs->outer_mom[sg.first_tensor], 16);
+        for (uint32_t k = 0; k < K && vec; ++k)
+            for (const Kind& kd : kinds)
+                if (kd.present && !aligned(buf_ptr(bufs, kd.id, (size_t)k * n_tensors + sg.first_tensor), 16))
+                    vec = false;
+        for (uint64_t off = 0; off < sg.numel; off += kChunkElems) {
+            const uint64_t len = sg.numel - off < kChunkElems ? sg.numel - off : kChunkElems;
+            chunks.push_back(Chunk{off, (uint32_t)len, (uint32_t)s | (vec ? kSegVecFlag : 0u)});
+        }
+    }
+    if (chunks.size() > 0x7FFFFFFFull / K) { delete ctx; return PALSGD_EUNSUPPORTED; }
+
+    // ---- one device blob: [DevState][chunks][7 pointer tables]
+    const size_t per_slot = (size_t)K * n_seg * sizeof(void*);
+    const size_t per_seg = n_seg * sizeof(void*);
+    size_t off_state = 0;
+    size_t off_chunks = round_up(sizeof(DevState), 256);
+    size_t off_tabs = round_up(off_chunks + chunks.size() * sizeof(Chunk), 256);
+    const size_t total = off_tabs + 5 * round_up(per_slot, 256) + 2 * round_up(per_seg, 256) + 256;
+    std::vector<char> host(total, 0);
+    DevState hs{};
+    for (uint32_t k = 0; k < kMaxWorkers; ++k) { hs.pow1[k] = 1.0; hs.pow2[k] = 1.0; }
+    std::memcpy(host.data() + off_state, &hs, sizeof(hs));
+    if (!chunks.empty()) std::memcpy(host.data() + off_chunks, chunks.data(), chunks.size() * sizeof(Chunk));
+
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (cudaMalloc(&ctx->d_blob, total) != cudaSuccess) {
+        cudaError_t e = cudaGetLastError();
+        g_noctx_err = std::string("cudaMalloc: ") + cudaGetErrorString(e);
+        delete ctx;
+        return e == cudaErrorMemoryAllocation ? PALSGD_ENOMEM : PALSGD_ECUDA;
+    }
+    char* d = static_cast<char*>(ctx->d_blob);
+    size_t cur = off_tabs;
+    auto fill_slot_table = [&](int kind) -> void* {
+        void** h = reinterpret_cast<void**>(host.data() + cur);
+        for (uint32_t k = 0; k < K; ++k)
+            for (size_t sgi = 0; sgi < n_seg; ++sgi)
+                h[(size_t)k * n_seg + sgi] =
+                    const_cast<void*>(buf_ptr(bufs, kind, (size_t)k * n_tensors + ctx->segs[sgi].first_tensor));
+        void* dev = d + cur;
+        cur += round_up(per_slot, 256);
+        return dev;
+    };
+    auto fill_seg_table = [&](float* const* src) -> void* {
+        void** h = reinterpret_cast<void**>(host.data() + cur);
+        for (size_t sgi = 0; sgi < n_seg; ++sgi) h[sgi] = src[ctx->segs[sgi].first_tensor];
+        void* dev = d + cur;
+        cur += round_up(per_seg, 256);
+        return dev;
+    };
+    Tables& tb = ctx->tb;
+    tb.st = reinterpret_cast<DevState*>(d + off_state);
+    tb.chunks = reinterpret_cast<const Chunk*>(d + off_chunks);
+    tb.n_chunks = (uint32_t)chunks.size();
+    tb.n_seg = (uint32_t)n_seg;
+    tb.K = K;
+    void* t_param = fill_slot_table(0);
+    tb.grad = static_cast<const void* const*>(fill_slot_table(1));
+    void* t_master = bf ? fill_slot_table(2) : nullptr;
+    tb.m = static_cast<float* const*>(fill_slot_table(3));
+    tb.v = adam ? static_cast<float* const*>(fill_slot_table(4)) : nullptr;
+    tb.global = static_cast<float* const*>(fill_seg_table(bufs->global));
+    tb.outer_mom = static_cast<float* const*>(fill_seg_table(bufs->outer_mom));
+    tb.xf = static_cast<float* const*>(bf ? t_master : t_param);
+    tb.xw = bf ? static_cast<__nv_bfloat16* const*>(t_param) : nullptr;
+
+    cudaError_t e = cudaMemcpyAsync(ctx->d_blob, host.data(), total, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);      // `host` is pageable and dies with this scope
+    if (e != cudaSuccess) { rc = cuda_fail(nullptr, e, "table upload"); cudaFree(ctx->d_blob); delete ctx; return rc; }
+
+    if (tb.n_chunks > 0) {
+        const OuterArgs oa = outer_args(ctx);
+        const unsigned grid = grid_for(tb.n_chunks, 0);
+        rc = launch_checked(ctx, [&] {
+            if (bf) palsgd_init_kernel<1><<<grid, kThreads, 0, s>>>(oa, adam ? 1 : 0);
+            else    palsgd_init_kernel<0><<<grid, kThreads, 0, s>>>(oa, adam ? 1 : 0);
+        });
+        if (rc) { g_noctx_err = ctx->cuda_err; cudaFree(ctx->d_blob); delete ctx; return rc; }
+    }
+    *out = ctx;
+    return PALSGD_OK;
+}
+
+// ------------------------------------------------------------------------- steps
+
+extern "C" int palsgd_inner_step(palsgd_ctx* ctx, double lr_t, double eta_t, void* stream)
+{
+    if (!ctx) return PALSGD_EINVAL;
+    if (!finite_nonneg(lr_t) || !finite_nonneg(eta_t)) return PALSGD_EINVAL;
+    const palsgd_config& c = ctx->cfg;
+    InnerArgs a{};
+    a.tb = ctx->tb;
+    a.seed = c.seed;
+    a.thr = ctx->thr;
+    a.beta1 = c.beta1;
+    a.beta2 = c.beta2;
+    // The coefficient of a branch that p rules out is never formed (p = 0: no pull; p = 1: no gradient step).
+    const double lr_d = c.p < 1.0 ? lr_t / (1.0 - c.p) : 0.0;
+    a.lr = (float)lr_d;
+    a.beta_pull = c.p > 0.0 ? (float)(lr_t * eta_t / c.p) : 0.0f;
+    a.b1 = (float)c.beta1;
+    a.b2 = (float)c.beta2;
+    a.omb1 = (float)(1.0 - c.beta1);
+    a.omb2 = (float)(1.0 - c.beta2);
+    a.eps = (float)c.eps;
+    a.decay = (float)(1.0 - lr_d * c.weight_decay);
+    a.mu = (float)c.momentum;
+    a.wd = (float)c.weight_decay;
+    int rc = launch_inner(ctx, a, static_cast<cudaStream_t>(stream));
+    if (rc) return rc;
+    ctx->t += 1;
+    return PALSGD_OK;
+}
+
+extern "C" int palsgd_pseudo_sync(palsgd_ctx* ctx, uint64_t worker_mask, double beta, void* stream)
+{
+    if (!ctx || !std::isfinite(beta)) return PALSGD_EINVAL;
+    const uint32_t K = ctx->cfg.K;
+    if (K < 64 && (worker_mask >> K) != 0) return PALSGD_EINVAL;
+    if (worker_mask == 0 || ctx->tb.n_chunks == 0) return PALSGD_OK;
+    PullArgs a{};
+    a.tb = ctx->tb;
+    a.mask = worker_mask;
+    a.beta = (float)beta;
+    const unsigned grid = grid_for((uint64_t)ctx->tb.n_chunks * K, ctx->grid_cap_inner);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const bool bf = ctx->cfg.precision == PALSGD_PREC_BF16_MASTER;
+    return launch_checked(ctx, [&] {
+        if (bf) palsgd_pull_kernel<1, 2><<<grid, kThreads, 0, s>>>(a);
+        else    palsgd_pull_kernel<0, 4><<<grid, kThreads, 0, s>>>(a);
+    });
+}
+
+extern "C" int palsgd_outer_sync(palsgd_ctx* ctx, void* stream)
+{
+    if (!ctx) return PALSGD_EINVAL;
+    if (ctx->tb.n_chunks > 0) {
+        const OuterArgs a = outer_args(ctx);
+        const unsigned grid = grid_for(ctx->tb.n_chunks, ctx->grid_cap_outer);
+        cudaStream_t s = static_cast<cudaStream_t>(stream);
+        const bool bf = ctx->cfg.precision == PALSGD_PREC_BF16_MASTER;
+        int rc = launch_checked(ctx, [&] {
+            if (bf) palsgd_outer_kernel<1><<<grid, kThreads, 0, s>>>(a);
+            else    palsgd_outer_kernel<0><<<grid, kThreads, 0, s>>>(a);
+        });
+        if (rc) return rc;
+    }
+    ctx->n_outer += 1;
+    return PALSGD_OK;
+}
+
+extern "C" int palsgd_step(palsgd_ctx* ctx, double lr_t, double eta_t, void* stream)
+{
+    int rc = palsgd_inner_step(ctx, lr_t, eta_t, stream);
+    if (rc) return rc;
+    if (ctx->t % ctx->cfg.H == 0) rc = palsgd_outer_sync(ctx, stream);
+    return rc;
+}
+
+extern "C" int palsgd_step_host(palsgd_ctx* ctx, const void* const* h_grad, double lr_t, double eta_t,
+                                float* const* h_global, uint8_t* h_decisions, int* synced, void* stream)
+{
+    if (!ctx || !h_grad) return PALSGD_EINVAL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t n = ctx->n_tensors;
+    const size_t gs = elem_size_param(ctx->cfg.precision);
+    // host -> device gradients; tensors adjacent on both sides travel as one copy
+    for (uint32_t k = 0; k < ctx->cfg.K; ++k) {
+        for (const Segment& sg : ctx->segs) {
+            size_t j = sg.first_tensor;
+            const size_t end = sg.first_tensor + sg.n_tensors;
+            while (j < end) {
+                const size_t idx = (size_t)k * n + j;
+                const char* src = static_cast<const char*>(h_grad[idx]);
+                if (!src) return PALSGD_EINVAL;
+                size_t bytes = ctx->numel[j] * gs;
+                size_t j2 = j + 1;
+                while (j2 < end && static_cast<const char*>(h_grad[(size_t)k * n + j2]) == src + bytes) {
+                    bytes += ctx->numel[j2] * gs;
+                    ++j2;
+                }
+                if (bytes)
+                    PALSGD_CUDA(ctx, cudaMemcpyAsync(const_cast<void*>(ctx->h_grad_dev[idx]), src, bytes,
+                                                     cudaMemcpyHostToDevice, s));
+                j = j2;
+            }
+        }
+    }
+    int rc = palsgd_inner_step(ctx, lr_t, eta_t, stream);
+    if (rc) return rc;
+    const bool sync_now = ctx->t % ctx->cfg.H == 0;
+    if (sync_now) { rc = palsgd_outer_sync(ctx, stream); if (rc) return rc; }
+    if (synced) *synced = sync_now ? 1 : 0;
+    if (h_decisions)
+        PALSGD_CUDA(ctx, cudaMemcpyAsync(h_decisions, ctx->tb.st->last_b, ctx->cfg.K, cudaMemcpyDeviceToHost, s));
+    if (sync_now && h_global) {
+        for (const Segment& sg : ctx->segs) {
+            size_t j = sg.first_tensor;
+            const size_t end = sg.first_tensor + sg.n_tensors;
+            while (j < end) {
+                char* dst = reinterpret_cast<char*>(h_global[j]);
+                if (!dst) return PALSGD_EINVAL;
+                size_t bytes = ctx->numel[j] * 4;
+                size_t j2 = j + 1;
+                while (j2 < end && reinterpret_cast<char*>(h_global[j2]) == dst + bytes) {
+                    bytes += ctx->numel[j2] * 4;
+                    ++j2;
+                }
+                if (bytes)
+                    PALSGD_CUDA(ctx, cudaMemcpyAsync(dst, ctx->h_global_dev[j], bytes, cudaMemcpyDeviceToHost, s));
+                j = j2;
+            }
+        }
+    }
+    PALSGD_CUDA(ctx, cudaStreamSynchronize(s));
+    return PALSGD_OK;
+}
+
+// ------------------------------------------------------------------------- counters
+
+extern "C" int palsgd_get_counters(palsgd_ctx* ctx, uint64_t* t, uint64_t* s_k, uint64_t* n_outer,
+                                   uint8_t* last_b, void* stream)
+{
+    if (!ctx) return PALSGD_EINVAL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    DevState hs;
+    PALSGD_CUDA(ctx, cudaMemcpyAsync(&hs, ctx->tb.st, sizeof(hs), cudaMemcpyDeviceToHost, s));
+    PALSGD_CUDA(ctx, cudaStreamSynchronize(s));
+    if (t) *t = hs.t;
+    if (n_outer) *n_outer = ctx->n_outer;
+    for (uint32_t k = 0; k < ctx->cfg.K; ++k) {
+        if (s_k) s_k[k] = hs.s[k];
+        if (last_b) last_b[k] = hs.last_b[k];
+    }
+    return hs.t == ctx->t ? PALSGD_OK : PALSGD_ESTATE;
+}
+
+extern "C" int palsgd_set_counters(palsgd_ctx* ctx, uint64_t t, const uint64_t* s_k, uint64_t n_outer,
+                                   void* stream)
+{
+    if (!ctx || !s_k) return PALSGD_EINVAL;
+    for (uint32_t k = 0; k < ctx->cfg.K; ++k)
+        if (s_k[k] > t) return PALSGD_EINVAL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    DevState hs{};
+    hs.t = t;
+    for (uint32_t k = 0; k < kMaxWorkers; ++k) {
+        hs.pow1[k] = 1.0; hs.pow2[k] = 1.0;
+        if (k < ctx->cfg.K) {
+            hs.s[k] = s_k[k];
+            for (uint64_t i = 0; i < s_k[k]; ++i) {      // the same running products the kernels form
+                hs.pow1[k] *= ctx->cfg.beta1;
+                hs.pow2[k] *= ctx->cfg.beta2;
+                if (hs.pow1[k] == 0.0 && hs.pow2[k] == 0.0) break;
+            }
+        }
+    }
+    PALSGD_CUDA(ctx, cudaMemcpyAsync(ctx->tb.st, &hs, sizeof(hs), cudaMemcpyHostToDevice, s));
+    PALSGD_CUDA(ctx, cudaStreamSynchronize(s));          // hs lives on this stack frame
+    ctx->t = t;
+    ctx->n_outer = n_outer;
+    return PALSGD_OK;
+}
+
+extern "C" int palsgd_get_launch_count(palsgd_ctx* ctx, uint64_t* n_launches)
+{
+    if (!ctx || !n_launches) return PALSGD_EINVAL;
+    *n_launches = ctx->launches;
+    return PALSGD_OK;
+}
+
+extern "C" int palsgd_set_tuning(palsgd_ctx* ctx, int knob, int64_t value)
+{
+    if (!ctx || value < 0 || value > 0x7FFFFFFF) return PALSGD_EINVAL;
+    switch (knob) {
+        case PALSGD_TUNE_INNER_GRID_CAP: ctx->grid_cap_inner = (int)value; return PALSGD_OK;
+        case PALSGD_TUNE_OUTER_GRID_CAP: ctx->grid_cap_outer = (int)value; return PALSGD_OK;
+        default: return PALSGD_EINVAL;
+    }
+}
+
+// ------------------------------------------------------------------------- pure host helpers
+
+extern "C" int palsgd_decision(uint64_t seed, uint64_t t, uint32_t k, double p)
+{
+    if (!(p >= 0.0 && p <= 1.0) || k >= PALSGD_MAX_WORKERS) return PALSGD_EINVAL;
+    return draw_pull(seed, t, k, threshold_of(p)) ? 1 : 0;
+}
+
+extern "C" const char* palsgd_strerror(int status)
+{
+    switch (status) {
+        case PALSGD_OK: return "ok";
+        case PALSGD_EINVAL: return "invalid argument";
+        case PALSGD_EALIGN: return "pointer not aligned to its element size";
+        case PALSGD_ECUDA: return "CUDA error";
+        case PALSGD_ESTATE: return "call not valid in this state";
+        case PALSGD_ENOMEM: return "out of memory";
+        case PALSGD_EUNSUPPORTED: return "unsupported combination";
+        default: return "unknown status";
+    }
+}
+
+extern "C" const char* palsgd_last_cuda_error(palsgd_ctx* ctx)
+{
+    return ctx ? ctx->cuda_err.c_str() : g_noctx_err.c_str();
+}
+
+extern "C" void palsgd_destroy(palsgd_ctx* ctx)
+{
+    if (!ctx) return;
+    if (ctx->d_blob) cudaFree(ctx->d_blob);
+    delete ctx;
+}

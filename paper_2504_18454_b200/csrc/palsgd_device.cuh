@@ -1,0 +1,76 @@
+// Device-side data structures shared by the PALSGD kernels and the host controller.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace palsgd {
+
+constexpr uint32_t kMaxWorkers  = 64;      // K <= 64 (worker masks are 64-bit)
+constexpr uint32_t kThreads     = 256;     // threads per CTA of every kernel here
+constexpr uint32_t kChunkElems  = 4096;    // elements per work item (one slot, one chunk)
+constexpr uint32_t kSegVecFlag  = 0x80000000u;   // Chunk::seg bit: 16-byte vector path allowed
+
+// One work unit of the multi-tensor launch: `len` consecutive elements of
+// segment `seg` starting at element `off`.  A segment is a maximal run of the
+// caller's tensors that are adjacent in memory in every buffer.
+struct Chunk {
+    uint64_t off;
+    uint32_t len;
+    uint32_t seg;        // segment index | kSegVecFlag
+};
+
+// Device-resident counters: the kernels read them and the last CTA of an inner
+// step advances them, so that a sequence of steps needs no host interaction
+// (and can be captured in a CUDA graph).
+struct DevState {
+    unsigned long long t;                    // completed inner steps (Algorithm 1's t)
+    unsigned long long s[kMaxWorkers];       // gradient steps taken by worker k
+    double             pow1[kMaxWorkers];    // beta1^s_k  (running product, binary64)
+    double             pow2[kMaxWorkers];    // beta2^s_k
+    unsigned int       done;                 // CTAs that finished the current inner launch
+    unsigned int       pad_;
+    unsigned char      last_b[kMaxWorkers];  // decisions of the latest inner step
+};
+
+// Device pointer tables, indexed [k * n_seg + seg] (per-slot) or [seg].
+struct Tables {
+    const Chunk*        chunks;
+    uint32_t            n_chunks;
+    uint32_t            n_seg;
+    uint32_t            K;
+    uint32_t            pad_;
+    float* const*       xf;         // fp32 model of slot k: params (FP32) or master (BF16_MASTER)
+    __nv_bfloat16* const* xw;       // bf16 working params (BF16_MASTER) else nullptr
+    const void* const*  grad;       // float or bf16 gradients
+    float* const*       m;
+    float* const*       v;          // nullptr table entries for SGD
+    float* const*       global;     // [n_seg]
+    float* const*       outer_mom;  // [n_seg]
+    DevState*           st;
+};
+
+struct InnerArgs {
+    Tables   tb;
+    uint64_t seed;
+    uint64_t thr;          // floor(p * 2^32): pull iff Philox word < thr
+    double   beta1, beta2; // binary64 decay rates for the running products
+    float    lr;           // fl32(alpha_t / (1 - p))
+    float    beta_pull;    // fl32(alpha_t * eta_t / p)
+    float    b1, b2, omb1, omb2, eps, decay;   // AdamW scalars, each rounded once from binary64
+    float    mu, wd;       // momentum SGD scalars
+};
+
+struct PullArgs {
+    Tables   tb;
+    uint64_t mask;         // workers to pull
+    float    beta;
+};
+
+struct OuterArgs {
+    Tables tb;
+    float  mu, lr, Kf;
+    int    nesterov;
+};
+
+}  // namespace palsgd

@@ -1,0 +1,554 @@
+// PALSGD kernels for sm_100a: fused inner step (branch draw + AdamW / momentum
+// SGD / pull), forced pull, outer sync (K-way average + Nesterov + broadcast),
+// and set-up.  All of them are HBM-bandwidth-bound streaming kernels: 128-bit
+// coalesced accesses, enough independent loads in flight per thread to cover
+// DRAM latency, streaming cache hints on data that is touched once per launch.
+//
+// Every element operation is written with the round-to-nearest intrinsics
+// (__fmul_rn, __fadd_rn, ...): they are single IEEE binary32 operations that
+// the compiler never fuses into a multiply-add, whatever flags are in force.
+#pragma once
+#include "palsgd_device.cuh"
+#include "palsgd_philox.cuh"
+
+namespace palsgd {
+
+// ---------------------------------------------------------------- element math
+
+struct AdamScalars { float b1, b2, omb1, omb2, bc1, bc2, decay, lr, eps; };
+struct SgdScalars  { float mu, wd, lr; };
+
+// AdamW with decoupled decay and bias correction (gradient branch, Eq. (1)).
+__device__ __forceinline__ void adamw_elem(float g, float& x, float& m, float& v, const AdamScalars& s)
+{
+    m = __fadd_rn(__fmul_rn(s.b1, m), __fmul_rn(s.omb1, g));
+    v = __fadd_rn(__fmul_rn(s.b2, v), __fmul_rn(s.omb2, __fmul_rn(g, g)));
+    const float mh = __fdiv_rn(m, s.bc1);
+    const float vh = __fdiv_rn(v, s.bc2);
+    x = __fmul_rn(x, s.decay);
+    x = __fsub_rn(x, __fmul_rn(s.lr, __fdiv_rn(mh, __fadd_rn(__fsqrt_rn(vh), s.eps))));
+}
+
+// Momentum SGD, L2 decay folded into the gradient (gradient branch, Eq. (1)).
+__device__ __forceinline__ void sgdm_elem(float g, float& x, float& buf, const SgdScalars& s)
+{
+    const float gp = __fadd_rn(g, __fmul_rn(s.wd, x));
+    buf = __fadd_rn(__fmul_rn(s.mu, buf), gp);
+    x = __fsub_rn(x, __fmul_rn(s.lr, buf));
+}
+
+// Pseudo-synchronisation (Eq. (2)): x <- x - beta (x - x_g).
+__device__ __forceinline__ float pull_elem(float x, float xg, float beta)
+{
+    return __fsub_rn(x, __fmul_rn(beta, __fsub_rn(x, xg)));
+}
+
+__device__ __forceinline__ float bf16_bits_to_f32(uint32_t h16) { return __uint_as_float(h16 << 16); }
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
+{
+    const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);      // RNE, .x in the low half
+    return *reinterpret_cast<const uint32_t*>(&v);
+}
+
+// streaming (touched once per launch) 128-bit accesses
+__device__ __forceinline__ float4 ld_stream(const float4* p) { return __ldcs(p); }
+__device__ __forceinline__ uint4  ld_stream(const uint4* p)  { return __ldcs(p); }
+__device__ __forceinline__ uint2  ld_stream(const uint2* p)  { return __ldcs(p); }
+__device__ __forceinline__ void   st_stream(float4* p, float4 v) { __stcs(p, v); }
+__device__ __forceinline__ void   st_stream(uint4* p, uint4 v)   { __stcs(p, v); }
+__device__ __forceinline__ void   st_stream(uint2* p, uint2 v)   { __stcs(p, v); }
+
+#define PALSGD_FOR4(EXPR)  { constexpr int c = 0; EXPR; } { constexpr int c = 1; EXPR; } \
+                           { constexpr int c = 2; EXPR; } { constexpr int c = 3; EXPR; }
+__device__ __forceinline__ float& comp(float4& a, int c) { return c == 0 ? a.x : c == 1 ? a.y : c == 2 ? a.z : a.w; }
+__device__ __forceinline__ float  compv(const float4& a, int c) { return c == 0 ? a.x : c == 1 ? a.y : c == 2 ? a.z : a.w; }
+
+// ---------------------------------------------------------------- fp32 chunk bodies
+
+// U independent 128-bit loads per stream are issued before any arithmetic.
+template <int U>
+__device__ __forceinline__ void adamw_chunk_f32(const float* __restrict__ g, float* __restrict__ x,
+                                                float* __restrict__ m, float* __restrict__ v,
+                                                uint32_t len, const AdamScalars& s)
+{
+    const uint32_t n4 = len >> 2;
+    const float4* g4 = reinterpret_cast<const float4*>(g);
+    float4* x4 = reinterpret_cast<float4*>(x);
+    float4* m4 = reinterpret_cast<float4*>(m);
+    float4* v4 = reinterpret_cast<float4*>(v);
+    for (uint32_t base = 0; base < n4; base += kThreads * U) {
+        float4 G[U], X[U], M[U], V[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const uint32_t i = base + u * kThreads + threadIdx.x;
+            if (i < n4) { G[u] = ld_stream(g4 + i); X[u] = ld_stream(x4 + i);
+                          M[u] = ld_stream(m4 + i); V[u] = ld_stream(v4 + i); }
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const uint32_t i = base + u * kThreads + threadIdx.x;
+            if (i < n4) {
+                PALSGD_FOR4(adamw_elem(compv(G[u], c), comp(X[u], c), comp(M[u], c), comp(V[u], c), s))
+                st_stream(x4 + i, X[u]); st_stream(m4 + i, M[u]); st_stream(v4 + i, V[u]);
+            }
+        }
+    }
+    const uint32_t i = (n4 << 2) + threadIdx.x;
+    if (i < len) { float xi = x[i], mi = m[i], vi = v[i]; adamw_elem(g[i], xi, mi, vi, s);
+                   x[i] = xi; m[i] = mi; v[i] = vi; }
+}
+
+template <int U>
+__device__ __forceinline__ void sgdm_chunk_f32(const float* __restrict__ g, float* __restrict__ x,
+                                               float* __restrict__ buf, uint32_t len, const SgdScalars& s)
+{
+    const uint32_t n4 = len >> 2;
+    const float4* g4 = reinterpret_cast<const float4*>(g);
+    float4* x4 = reinterpret_cast<float4*>(x);
+    float4* b4 = reinterpret_cast<float4*>(buf);
+    for (uint32_t base = 0; base < n4; base += kThreads * U) {
+        float4 G[U], X[U], B[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const uint32_t i = base + u * kThreads + threadIdx.x;
+            if (i < n4) { G[u] = ld_stream(g4 + i); X[u] = ld_stream(x4 + i); B[u] = ld_stream(b4 + i); }
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const uint32_t i = base + u * kThreads + threadIdx.x;
+            if (i < n4) {
+                PALSGD_FOR4(sgdm_elem(compv(G[u], c), comp(X[u], c), comp(B[u], c), s))
+                st_stream(x4 + i, X[u]); st_stream(b4 + i, B[u]);
+            }
+        }
+    }
+    const uint32_t i = (n4 << 2) + threadIdx.x;
+    if (i < len) { float xi = x[i], bi = buf[i]; sgdm_elem(g[i], xi, bi, s); x[i] = xi; buf[i] = bi; }
+}
+
+// x_g is read with the default policy: slots that pull in the same step share it through L2.
+template <int U>
+__device__ __forceinline__ void pull_chunk_f32(float* __restrict__ x, const float* __restrict__ xg,
+                                               uint32_t len, float beta)
+{
+    const uint32_t n4 = len >> 2;
+    float4* x4 = reinterpret_cast<float4*>(x);
+    const float4* q4 = reinterpret_cast<const float4*>(xg);
+    for (uint32_t base = 0; base < n4; base += kThreads * U) {
+        float4 X[U], Q[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const uint32_t i = base + u * kThreads + threadIdx.x;
+            if (i < n4) { X[u] = ld_stream(x4 + i); Q[u] = __ldg(q4 + i); }
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const uint32_t i = base + u * kThreads + threadIdx.x;
+            if (i < n4) {
+                PALSGD_FOR4(comp(X[u], c) = pull_elem(compv(X[u], c), compv(Q[u], c), beta))
+                st_stream(x4 + i, X[u]);
+            }
+        }
+    }
+    const uint32_t i = (n4 << 2) + threadIdx.x;
+    if (i < len) x[i] = pull_elem(x[i], xg[i], beta);
+}
+
+// ---------------------------------------------------------------- bf16 + fp32-master chunk bodies
+// Groups of 8 elements: one 128-bit load of bf16 gradients, two per fp32 stream.
+
+__device__ __forceinline__ void unpack8(const uint4& h, float (&f)[8])
+{
+    f[0] = bf16_bits_to_f32(h.x & 0xFFFFu); f[1] = __uint_as_float(h.x & 0xFFFF0000u);
+    f[2] = bf16_bits_to_f32(h.y & 0xFFFFu); f[3] = __uint_as_float(h.y & 0xFFFF0000u);
+    f[4] = bf16_bits_to_f32(h.z & 0xFFFFu); f[5] = __uint_as_float(h.z & 0xFFFF0000u);
+    f[6] = bf16_bits_to_f32(h.w & 0xFFFFu); f[7] = __uint_as_float(h.w & 0xFFFF0000u);
+}
+
+__device__ __forceinline__ uint4 pack8(const float4& a, const float4& b)
+{
+    return make_uint4(pack_bf16x2(a.x, a.y), pack_bf16x2(a.z, a.w),
+                      pack_bf16x2(b.x, b.y), pack_bf16x2(b.z, b.w));
+}
+
+template <int U>
+__device__ __forceinline__ void adamw_chunk_bf16(const __nv_bfloat16* __restrict__ g,
+                                                 __nv_bfloat16* __restrict__ w, float* __restrict__ x,
+                                                 float* __restrict__ m, float* __restrict__ v,
+                                                 uint32_t len, const AdamScalars& s)
+{
+    const uint32_t n8 = len >> 3;
+    const uint4* g8 = reinterpret_cast<const uint4*>(g);
+    uint4* w8 = reinterpret_cast<uint4*>(w);
+    float4* x4 = reinterpret_cast<float4*>(x);
+    float4* m4 = reinterpret_cast<float4*>(m);
+    float4* v4 = reinterpret_cast<float4*>(v);
+    for (uint32_t base = 0; base < n8; base += kThreads * U) {
+        uint4 G[U]; float4 X[U][2], M[U][2], V[U][2];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const uint32_t i = base + u * kThreads + threadIdx.x;
+            if (i < n8) {
+                G[u] = ld_stream(g8 + i);
+                X[u][0] = ld_stream(x4 + 2 * i); X[u][1] = ld_stream(x4 + 2 * i + 1);
+                M[u][0] = ld_stream(m4 + 2 * i); M[u][1] = ld_stream(m4 + 2 * i + 1);
+                V[u][0] = ld_stream(v4 + 2 * i); V[u][1] = ld_stream(v4 + 2 * i + 1);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const uint32_t i = base + u * kThreads + threadIdx.x;
+            if (i < n8) {
+                float gf[8]; unpack8(G[u], gf);
+                PALSGD_FOR4(adamw_elem(gf[c],     comp(X[u][0], c), comp(M[u][0], c), comp(V[u][0], c), s))
+                PALSGD_FOR4(adamw_elem(gf[4 + c], comp(X[u][1], c), comp(M[u][1], c), comp(V[u][1], c), s))
+                st_stream(x4 + 2 * i, X[u][0]); st_stream(x4 + 2 * i + 1, X[u][1]);
+                st_stream(m4 + 2 * i, M[u][0]); st_stream(m4 + 2 * i + 1, M[u][1]);
+                st_stream(v4 + 2 * i, V[u][0]); st_stream(v4 + 2 * i + 1, V[u][1]);
+                st_stream(w8 + i, pack8(X[u][0], X[u][1]));
+            }
+        }
+    }
+    const uint32_t i = (n8 << 3) + threadIdx.x;
+    if (i < len) { float xi = x[i], mi = m[i], vi = v[i];
+                   adamw_elem(__bfloat162float(g[i]), xi, mi, vi, s);
+                   x[i] = xi; m[i] = mi; v[i] = vi; w[i] = __float2bfloat16_rn(xi); }
+}
+
+template <int U>
+__device__ __forceinline__ void sgdm_chunk_bf16(const __nv_bfloat16* __restrict__ g,
+                                                __nv_bfloat16* __restrict__ w, float* __restrict__ x,
+                                                float* __restrict__ buf, uint32_t len, const SgdScalars& s)
+{
+    const uint32_t n8 = len >> 3;
+    const uint4* g8 = reinterpret_cast<const uint4*>(g);
+    uint4* w8 = reinterpret_cast<uint4*>(w);
+    float4* x4 = reinterpret_cast<float4*>(x);
+    float4* b4 = reinterpret_cast<float4*>(buf);
+    for (uint32_t base = 0; base < n8; base += kThreads * U) {
+        uint4 G[U]; float4 X[U][2], B[U][2];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const uint32_t i = base + u * kThreads + threadIdx.x;
+            if (i < n8) {
+                G[u] = ld_stream(g8 + i);
+                X[u][0] = ld_stream(x4 + 2 * i); X[u][1] = ld_stream(x4 + 2 * i + 1);
+                B[u][0] = ld_stream(b4 + 2 * i); B[u][1] = ld_stream(b4 + 2 * i + 1);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const uint32_t i = base + u * kThreads + threadIdx.x;
+            if (i < n8) {
+                float gf[8]; unpack8(G[u], gf);
+                PALSGD_FOR4(sgdm_elem(gf[c],     comp(X[u][0], c), comp(B[u][0], c), s))
+                PALSGD_FOR4(sgdm_elem(gf[4 + c], comp(X[u][1], c), comp(B[u][1], c), s))
+                st_stream(x4 + 2 * i, X[u][0]); st_stream(x4 + 2 * i + 1, X[u][1]);
+                st_stream(b4 + 2 * i, B[u][0]); st_stream(b4 + 2 * i + 1, B[u][1]);
+                st_stream(w8 + i, pack8(X[u][0], X[u][1]));
+            }
+        }
+    }
+    const uint32_t i = (n8 << 3) + threadIdx.x;
+    if (i < len) { float xi = x[i], bi = buf[i]; sgdm_elem(__bfloat162float(g[i]), xi, bi, s);
+                   x[i] = xi; buf[i] = bi; w[i] = __float2bfloat16_rn(xi); }
+}
+
+template <int U>
+__device__ __forceinline__ void pull_chunk_bf16(__nv_bfloat16* __restrict__ w, float* __restrict__ x,
+                                                const float* __restrict__ xg, uint32_t len, float beta)
+{
+    const uint32_t n8 = len >> 3;
+    uint4* w8 = reinterpret_cast<uint4*>(w);
+    float4* x4 = reinterpret_cast<float4*>(x);
+    const float4* q4 = reinterpret_cast<const float4*>(xg);
+    for (uint32_t base = 0; base < n8; base += kThreads * U) {
+        float4 X[U][2], Q[U][2];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const uint32_t i = base + u * kThreads + threadIdx.x;
+            if (i < n8) { X[u][0] = ld_stream(x4 + 2 * i); X[u][1] = ld_stream(x4 + 2 * i + 1);
+                          Q[u][0] = __ldg(q4 + 2 * i);      Q[u][1] = __ldg(q4 + 2 * i + 1); }
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const uint32_t i = base + u * kThreads + threadIdx.x;
+            if (i < n8) {
+                PALSGD_FOR4(comp(X[u][0], c) = pull_elem(compv(X[u][0], c), compv(Q[u][0], c), beta))
+                PALSGD_FOR4(comp(X[u][1], c) = pull_elem(compv(X[u][1], c), compv(Q[u][1], c), beta))
+                st_stream(x4 + 2 * i, X[u][0]); st_stream(x4 + 2 * i + 1, X[u][1]);
+                st_stream(w8 + i, pack8(X[u][0], X[u][1]));
+            }
+        }
+    }
+    const uint32_t i = (n8 << 3) + threadIdx.x;
+    if (i < len) { const float xi = pull_elem(x[i], xg[i], beta); x[i] = xi; w[i] = __float2bfloat16_rn(xi); }
+}
+
+// ---------------------------------------------------------------- scalar bodies (unaligned segments)
+
+template <int INNER, int PREC>
+__device__ __forceinline__ void grad_chunk_scalar(const void* g, __nv_bfloat16* w, float* x, float* m, float* v,
+                                                  uint32_t len, const AdamScalars& as, const SgdScalars& ss)
+{
+    for (uint32_t i = threadIdx.x; i < len; i += kThreads) {
+        const float gi = PREC ? __bfloat162float(static_cast<const __nv_bfloat16*>(g)[i])
+                              : static_cast<const float*>(g)[i];
+        float xi = x[i], mi = m[i];
+        if (INNER == 0) { float vi = v[i]; adamw_elem(gi, xi, mi, vi, as); v[i] = vi; }
+        else            { sgdm_elem(gi, xi, mi, ss); }
+        x[i] = xi; m[i] = mi;
+        if (PREC) w[i] = __float2bfloat16_rn(xi);
+    }
+}
+
+template <int PREC>
+__device__ __forceinline__ void pull_chunk_scalar(__nv_bfloat16* w, float* x, const float* xg, uint32_t len, float beta)
+{
+    for (uint32_t i = threadIdx.x; i < len; i += kThreads) {
+        const float xi = pull_elem(x[i], xg[i], beta);
+        x[i] = xi;
+        if (PREC) w[i] = __float2bfloat16_rn(xi);
+    }
+}
+
+// ---------------------------------------------------------------- dispatch of one work item
+
+template <int PREC, int U>
+__device__ __forceinline__ void pull_item(const Tables& tb, uint32_t k, const Chunk& ch, float beta)
+{
+    const uint32_t seg = ch.seg & ~kSegVecFlag;
+    const size_t   pi  = (size_t)k * tb.n_seg + seg;
+    float* x = tb.xf[pi] + ch.off;
+    const float* xg = tb.global[seg] + ch.off;
+    __nv_bfloat16* w = PREC ? tb.xw[pi] + ch.off : nullptr;
+    if (ch.seg & kSegVecFlag) {
+        if (PREC) pull_chunk_bf16<U>(w, x, xg, ch.len, beta);
+        else      pull_chunk_f32<U>(x, xg, ch.len, beta);
+    } else {
+        pull_chunk_scalar<PREC>(w, x, xg, ch.len, beta);
+    }
+}
+
+template <int INNER, int PREC, int U>
+__device__ __forceinline__ void grad_item(const Tables& tb, uint32_t k, const Chunk& ch,
+                                          const AdamScalars& as, const SgdScalars& ss)
+{
+    const uint32_t seg = ch.seg & ~kSegVecFlag;
+    const size_t   pi  = (size_t)k * tb.n_seg + seg;
+    float* x = tb.xf[pi] + ch.off;
+    float* m = tb.m[pi] + ch.off;
+    float* v = INNER == 0 ? tb.v[pi] + ch.off : nullptr;
+    if (PREC) {
+        const __nv_bfloat16* g = static_cast<const __nv_bfloat16*>(tb.grad[pi]) + ch.off;
+        __nv_bfloat16* w = tb.xw[pi] + ch.off;
+        if (ch.seg & kSegVecFlag) {
+            if (INNER == 0) adamw_chunk_bf16<U>(g, w, x, m, v, ch.len, as);
+            else            sgdm_chunk_bf16<U>(g, w, x, m, ch.len, ss);
+        } else {
+            grad_chunk_scalar<INNER, 1>(g, w, x, m, v, ch.len, as, ss);
+        }
+    } else {
+        const float* g = static_cast<const float*>(tb.grad[pi]) + ch.off;
+        if (ch.seg & kSegVecFlag) {
+            if (INNER == 0) adamw_chunk_f32<U>(g, x, m, v, ch.len, as);
+            else            sgdm_chunk_f32<U>(g, x, m, ch.len, ss);
+        } else {
+            grad_chunk_scalar<INNER, 0>(g, nullptr, x, m, v, ch.len, as, ss);
+        }
+    }
+}
+
+// ---------------------------------------------------------------- fused inner step
+// One launch per step of Algorithm 1's inner loop body.  Work item = (chunk c,
+// worker k), k fastest, so neighbouring CTAs that pull share x_g through L2.
+// Every CTA recomputes the K decisions of step t from the counter-based
+// stream; the last CTA to finish advances the device counters.
+
+template <int INNER, int PREC, int U>
+__global__ void __launch_bounds__(kThreads)
+palsgd_inner_kernel(const __grid_constant__ InnerArgs a)
+{
+    __shared__ unsigned char s_pull[kMaxWorkers];
+    __shared__ float s_bc1[kMaxWorkers], s_bc2[kMaxWorkers];
+
+    const Tables& tb = a.tb;
+    const uint32_t K = tb.K;
+    DevState* st = tb.st;
+    const unsigned long long t = st->t;
+
+    if (threadIdx.x < K) {
+        const uint32_t k = threadIdx.x;
+        const bool pull = draw_pull(a.seed, t, k, a.thr);
+        s_pull[k] = pull;
+        if (INNER == 0 && !pull) {                       // bias corrections for gradient step s_k + 1
+            s_bc1[k] = (float)(1.0 - st->pow1[k] * a.beta1);
+            s_bc2[k] = (float)(1.0 - st->pow2[k] * a.beta2);
+        }
+    }
+    __syncthreads();
+
+    const uint64_t n_items = (uint64_t)tb.n_chunks * K;
+    for (uint64_t item = blockIdx.x; item < n_items; item += gridDim.x) {
+        const uint32_t k = (uint32_t)(item % K);
+        const Chunk ch = tb.chunks[item / K];
+        if (s_pull[k]) {
+            pull_item<PREC, U>(tb, k, ch, a.beta_pull);
+        } else {
+            const AdamScalars as{a.b1, a.b2, a.omb1, a.omb2, s_bc1[k], s_bc2[k], a.decay, a.lr, a.eps};
+            const SgdScalars  ss{a.mu, a.wd, a.lr};
+            grad_item<INNER, PREC, U>(tb, k, ch, as, ss);
+        }
+    }
+
+    // ---- counter tick by the last CTA (all state reads above precede the atomic)
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        const unsigned int prev = atomicAdd(&st->done, 1u);
+        if (prev == gridDim.x - 1) {
+            for (uint32_t k = 0; k < K; ++k) {
+                const bool pull = s_pull[k];
+                st->last_b[k] = pull;
+                if (!pull) {
+                    st->s[k] += 1;
+                    if (INNER == 0) { st->pow1[k] *= a.beta1; st->pow2[k] *= a.beta2; }
+                }
+            }
+            st->t = t + 1;
+            st->done = 0;
+            __threadfence();
+        }
+    }
+}
+
+// ---------------------------------------------------------------- forced pull
+template <int PREC, int U>
+__global__ void __launch_bounds__(kThreads)
+palsgd_pull_kernel(const __grid_constant__ PullArgs a)
+{
+    const Tables& tb = a.tb;
+    const uint32_t K = tb.K;
+    const uint64_t n_items = (uint64_t)tb.n_chunks * K;
+    for (uint64_t item = blockIdx.x; item < n_items; item += gridDim.x) {
+        const uint32_t k = (uint32_t)(item % K);
+        if ((a.mask >> k) & 1ull) pull_item<PREC, U>(tb, k, tb.chunks[item / K], a.beta);
+    }
+}
+
+// ---------------------------------------------------------------- outer sync
+// Per element: average of the K slots in ascending k, outer gradient, (Nesterov)
+// momentum update, and the new global model written to x_g and to all K slots
+// (and K bf16 working copies) in the same pass.
+
+__device__ __forceinline__ float outer_elem(float sum, float Kf, float xg, float& u, float mu, float lr, int nesterov)
+{
+    const float xbar  = __fdiv_rn(sum, Kf);
+    const float delta = __fsub_rn(xg, xbar);
+    u = __fadd_rn(__fmul_rn(mu, u), delta);
+    const float step = nesterov ? __fadd_rn(delta, __fmul_rn(mu, u)) : u;
+    return __fsub_rn(xg, __fmul_rn(lr, step));
+}
+
+template <int PREC>
+__global__ void __launch_bounds__(kThreads)
+palsgd_outer_kernel(const __grid_constant__ OuterArgs a)
+{
+    __shared__ float* s_x[kMaxWorkers];
+    __shared__ __nv_bfloat16* s_w[kMaxWorkers];
+    const Tables& tb = a.tb;
+    const uint32_t K = tb.K;
+    constexpr int B = 8;                                   // slot loads issued together
+
+    for (uint32_t c = blockIdx.x; c < tb.n_chunks; c += gridDim.x) {
+        const Chunk ch = tb.chunks[c];
+        const uint32_t seg = ch.seg & ~kSegVecFlag;
+        __syncthreads();
+        if (threadIdx.x < K) {
+            const size_t pi = (size_t)threadIdx.x * tb.n_seg + seg;
+            s_x[threadIdx.x] = tb.xf[pi] + ch.off;
+            if (PREC) s_w[threadIdx.x] = tb.xw[pi] + ch.off;
+        }
+        __syncthreads();
+        float* xg = tb.global[seg] + ch.off;
+        float* um = tb.outer_mom[seg] + ch.off;
+
+        uint32_t done = 0;
+        if (ch.seg & kSegVecFlag) {
+            const uint32_t n4 = ch.len >> 2;
+            for (uint32_t i = threadIdx.x; i < n4; i += kThreads) {
+                const float4 Q = __ldcs(reinterpret_cast<const float4*>(xg) + i);
+                float4 Um = __ldcs(reinterpret_cast<const float4*>(um) + i);
+                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                for (uint32_t k0 = 0; k0 < K; k0 += B) {
+                    float4 R[B];
+#pragma unroll
+                    for (int j = 0; j < B; ++j)
+                        if (k0 + j < K) R[j] = __ldcs(reinterpret_cast<const float4*>(s_x[k0 + j]) + i);
+#pragma unroll
+                    for (int j = 0; j < B; ++j)
+                        if (k0 + j < K) {
+                            if (k0 + j == 0) acc = R[j];
+                            else { acc.x = __fadd_rn(acc.x, R[j].x); acc.y = __fadd_rn(acc.y, R[j].y);
+                                   acc.z = __fadd_rn(acc.z, R[j].z); acc.w = __fadd_rn(acc.w, R[j].w); }
+                        }
+                }
+                float4 N;
+                N.x = outer_elem(acc.x, a.Kf, Q.x, Um.x, a.mu, a.lr, a.nesterov);
+                N.y = outer_elem(acc.y, a.Kf, Q.y, Um.y, a.mu, a.lr, a.nesterov);
+                N.z = outer_elem(acc.z, a.Kf, Q.z, Um.z, a.mu, a.lr, a.nesterov);
+                N.w = outer_elem(acc.w, a.Kf, Q.w, Um.w, a.mu, a.lr, a.nesterov);
+                __stcs(reinterpret_cast<float4*>(xg) + i, N);
+                __stcs(reinterpret_cast<float4*>(um) + i, Um);
+                for (uint32_t k = 0; k < K; ++k) __stcs(reinterpret_cast<float4*>(s_x[k]) + i, N);
+                if (PREC) {
+                    const uint2 h = make_uint2(pack_bf16x2(N.x, N.y), pack_bf16x2(N.z, N.w));
+                    for (uint32_t k = 0; k < K; ++k) __stcs(reinterpret_cast<uint2*>(s_w[k]) + i, h);
+                }
+            }
+            done = n4 << 2;
+        }
+        for (uint32_t i = done + threadIdx.x; i < ch.len; i += kThreads) {
+            float sum = s_x[0][i];
+            for (uint32_t k = 1; k < K; ++k) sum = __fadd_rn(sum, s_x[k][i]);
+            float ui = um[i];
+            const float xn = outer_elem(sum, a.Kf, xg[i], ui, a.mu, a.lr, a.nesterov);
+            xg[i] = xn; um[i] = ui;
+            for (uint32_t k = 0; k < K; ++k) s_x[k][i] = xn;
+            if (PREC) { const __nv_bfloat16 h = __float2bfloat16_rn(xn);
+                        for (uint32_t k = 0; k < K; ++k) s_w[k][i] = h; }
+        }
+    }
+}
+
+// ---------------------------------------------------------------- set-up
+// x_g <- fixed-order mean of the slots, u <- 0, m, v <- 0, bf16 working <- RNE(master).
+template <int PREC>
+__global__ void __launch_bounds__(kThreads)
+palsgd_init_kernel(const __grid_constant__ OuterArgs a, int has_v)
+{
+    const Tables& tb = a.tb;
+    const uint32_t K = tb.K;
+    for (uint32_t c = blockIdx.x; c < tb.n_chunks; c += gridDim.x) {
+        const Chunk ch = tb.chunks[c];
+        const uint32_t seg = ch.seg & ~kSegVecFlag;
+        float* xg = tb.global[seg] + ch.off;
+        float* um = tb.outer_mom[seg] + ch.off;
+        for (uint32_t i = threadIdx.x; i < ch.len; i += kThreads) {
+            float sum = 0.f;
+            for (uint32_t k = 0; k < K; ++k) {
+                const size_t pi = (size_t)k * tb.n_seg + seg;
+                const float xi = tb.xf[pi][ch.off + i];
+                sum = k == 0 ? xi : __fadd_rn(sum, xi);
+                tb.m[pi][ch.off + i] = 0.f;
+                if (has_v) tb.v[pi][ch.off + i] = 0.f;
+                if (PREC) tb.xw[pi][ch.off + i] = __float2bfloat16_rn(xi);
+            }
+            xg[i] = __fdiv_rn(sum, a.Kf);
+            um[i] = 0.f;
+        }
+    }
+}
+
+}  // namespace palsgd

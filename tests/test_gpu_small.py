@@ -1,0 +1,206 @@
+"""GPU parity, small cases: the CUDA library against the CPU oracle, element by
+element, over shapes that span several chunks and ragged tails, both optimizers,
+both precisions, all three buffer layouts, and the degenerate settings."""
+import numpy as np
+import pytest
+import torch
+
+import workloads as W
+from workloads.configs import WorkloadConfig
+from _harness import GpuRun, compare_state, make_oracle
+
+pytestmark = pytest.mark.gpu
+
+RAGGED = [1, 3, 7, 1001, 4095, 4096, 4097, 0, 5, 12289, 8]     # > 6 chunks, odd tails, an empty tensor
+
+
+def _cfg(numel, **kw):
+    base = dict(name="t", shape=lambda: [], K=4, H=4, p=0.25, eta=16.0, lr=1e-3, T=10)
+    base.update(kw)
+    return WorkloadConfig(**base)
+
+
+def _x0(K, P, seed=1, same=False):
+    rng = np.random.default_rng(seed)
+    if same:
+        return np.tile((rng.standard_normal(P) * 0.02).astype(np.float32), (K, 1))
+    return (rng.standard_normal((K, P)) * 0.02).astype(np.float32)
+
+
+def _grads(cfg, P, t):
+    g = np.stack([W.grads_host(P, cfg.grad_seed, t, k, cfg.grad_std) for k in range(cfg.K)])
+    return W.bf16_bits_from_f32_host(g) if cfg.precision == 1 else g
+
+
+def _run_both(cfg, numel, layout, T=None, x0=None, check_every_step=True):
+    P = int(sum(numel))
+    x0 = _x0(cfg.K, P) if x0 is None else x0
+    gpu = GpuRun(cfg, x0, numel=numel, layout=layout)
+    orc = make_oracle(cfg, x0)
+    compare_state(gpu.state(), orc, exact=True)                   # init: mean, zeros, bf16 copy
+    for t in range(T if T is not None else cfg.T):
+        g = _grads(cfg, P, t)
+        gpu.set_grads(g)
+        gpu.step(cfg.lr, cfg.eta)
+        orc.step(g, cfg.lr, cfg.eta)
+        if check_every_step:
+            c = gpu.counters()
+            assert c["t"] == orc.t and c["n_outer"] == orc.n_outer
+            assert c["s"] == [int(v) for v in orc.s]              # bit-exact integer state
+            assert c["last_b"] == [int(v) for v in orc.last_b]
+    rep = compare_state(gpu.state(), orc, exact=True)
+    assert gpu.guards_intact()
+    return gpu, orc, rep
+
+
+@pytest.mark.parametrize("layout", ["arena", "separate", "misaligned"])
+@pytest.mark.parametrize("inner,precision", [(0, 0), (1, 0), (0, 1), (1, 1)])
+def test_ragged_tensor_list_matches_oracle(layout, inner, precision):
+    cfg = _cfg(RAGGED, inner=inner, precision=precision, momentum=0.9 if inner else 0.0,
+               weight_decay=1e-4 if inner else 0.01)
+    _run_both(cfg, RAGGED, layout)
+
+
+@pytest.mark.parametrize("K", [1, 2, 3, 8, 32, 64])
+def test_worker_counts(K):
+    numel = [4096 * 2 + 13]
+    cfg = _cfg(numel, K=K, H=3, T=7)
+    _run_both(cfg, numel, "arena")
+
+
+@pytest.mark.parametrize("numel", [[1], [3], [7], [4095], [4097], [0, 0, 2]])
+def test_tiny_and_edge_sizes(numel):
+    _run_both(_cfg(numel, K=3, H=2, T=5), numel, "separate")
+    _run_both(_cfg(numel, K=3, H=2, T=5, precision=1), numel, "arena")
+
+
+@pytest.mark.parametrize("p", [0.0, 1.0, 0.5])
+def test_extreme_probabilities(p):
+    numel = [5000]
+    gpu, orc, _ = _run_both(_cfg(numel, p=p, H=4, T=8), numel, "arena")
+    c = gpu.counters()
+    if p == 0.0:
+        assert c["s"] == [8] * 4             # never pulls: DiLoCo
+    if p == 1.0:
+        assert c["s"] == [0] * 4             # always pulls
+
+
+def test_plain_averaging_outer_and_momentum_without_nesterov():
+    numel = [9000]
+    _run_both(_cfg(numel, outer_lr=1.0, outer_momentum=0.0, outer_nesterov=False, H=3, T=6), numel, "arena")
+    _run_both(_cfg(numel, outer_lr=0.5, outer_momentum=0.8, outer_nesterov=False, H=3, T=6), numel, "arena")
+
+
+def test_h_equal_one_and_t_not_multiple_of_h():
+    numel = [4099]
+    _run_both(_cfg(numel, H=1, T=4), numel, "arena")
+    _run_both(_cfg(numel, H=5, T=7), numel, "arena")
+
+
+def test_slots_that_differ_at_start_get_the_fixed_order_mean():
+    numel = [6000]
+    cfg = _cfg(numel, K=5)
+    _run_both(cfg, numel, "arena", x0=_x0(5, 6000, seed=3, same=False), T=5)
+
+
+def test_large_pull_coefficient_is_not_clamped():
+    numel = [3000]
+    _run_both(_cfg(numel, eta=400.0, p=0.25, T=6), numel, "arena")      # beta = 1.6
+
+
+def test_separate_entry_points_inner_pull_outer():
+    numel = RAGGED
+    P = sum(numel)
+    for precision in (0, 1):
+        cfg = _cfg(numel, precision=precision, H=10**6)
+        x0 = _x0(cfg.K, P, seed=9)
+        gpu, orc = GpuRun(cfg, x0, numel=numel), make_oracle(cfg, x0)
+        for t in range(3):
+            g = _grads(cfg, P, t)
+            gpu.set_grads(g); gpu.inner_step(cfg.lr, cfg.eta); orc.inner_step(g, cfg.lr, cfg.eta)
+        gpu.pseudo_sync(0b0101, 0.3); orc.pseudo_sync(0b0101, 0.3)
+        compare_state(gpu.state(), orc, exact=True)
+        c = gpu.counters()
+        assert c["t"] == 3 and c["n_outer"] == 0 and c["s"] == [int(v) for v in orc.s]
+        gpu.outer_sync(); orc.outer_sync()
+        st = gpu.state()
+        compare_state(st, orc, exact=True)
+        for k in range(cfg.K):                                    # consensus, bitwise
+            assert np.array_equal(st["x"][k], st["xg"])
+        assert gpu.counters()["n_outer"] == 1
+        gpu.pseudo_sync(0, 0.3)                                   # empty mask: no-op
+        with pytest.raises(Exception):
+            gpu.pseudo_sync(1 << cfg.K, 0.3)                      # bit beyond K
+
+
+def test_checkpoint_resume_is_bit_exact():
+    numel = [10000]
+    cfg = _cfg(numel, H=4)
+    P = 10000
+    x0 = _x0(cfg.K, P, same=True)
+    a = GpuRun(cfg, x0, numel=numel)
+    for t in range(8):
+        a.set_grads(_grads(cfg, P, t)); a.step(cfg.lr, cfg.eta)
+    want = a.state()
+    b = GpuRun(cfg, x0, numel=numel)
+    for t in range(4):
+        b.set_grads(_grads(cfg, P, t)); b.step(cfg.lr, cfg.eta)
+    saved, cnt = b.state(), b.counters()
+    c = GpuRun(cfg, x0, numel=numel)                              # fresh context, restore, continue
+    for name, key in (("param", "x"), ("m", "m"), ("v", "v")):
+        c._write(name, saved[key])
+    c._write("global_", saved["xg"][None]); c._write("outer_mom", saved["u"][None])
+    c.lib.set_counters(cnt["t"], cnt["s"], cnt["n_outer"], c.stream)
+    for t in range(4, 8):
+        c.set_grads(_grads(cfg, P, t)); c.step(cfg.lr, cfg.eta)
+    got = c.state()
+    for k in want:
+        assert np.array_equal(want[k], got[k]), k
+    assert c.counters() == a.counters()
+
+
+def test_run_to_run_determinism_and_launch_shape_independence():
+    numel = RAGGED
+    P = sum(numel)
+    cfg = _cfg(numel, K=8, H=3, T=6)
+    x0 = _x0(cfg.K, P, same=True)
+    outs = []
+    for caps in (None, None, (7, 3), (148 * 4, 148)):
+        r = GpuRun(cfg, x0, numel=numel)
+        if caps:
+            r.lib.set_tuning(0, caps[0]); r.lib.set_tuning(1, caps[1])
+        for t in range(cfg.T):
+            r.set_grads(_grads(cfg, P, t)); r.step(cfg.lr, cfg.eta)
+        outs.append(r.state())
+        assert r.lib.get_launch_count() == 1 + cfg.T + cfg.T // cfg.H   # init + inner + outer
+    for o in outs[1:]:
+        for k in outs[0]:
+            assert np.array_equal(outs[0][k], o[k]), k
+
+
+def test_step_host_moves_gradients_and_results_through_host_buffers():
+    numel = [5000, 37, 4096]
+    P = sum(numel)
+    for precision in (0, 1):
+        cfg = _cfg(numel, precision=precision, H=2)
+        x0 = _x0(cfg.K, P, same=True)
+        gpu, orc = GpuRun(cfg, x0, numel=numel, layout="separate"), make_oracle(cfg, x0)
+        gdt = torch.int16 if precision else torch.float32
+        hg = torch.empty((cfg.K, P), dtype=gdt).pin_memory()
+        hx = torch.empty(P, dtype=torch.float32).pin_memory()
+        hb = torch.zeros(cfg.K, dtype=torch.uint8).pin_memory()
+        starts = np.concatenate([[0], np.cumsum(numel)])
+        es = hg.element_size()
+        gp = gpu.lib.make_ptr_array([hg.data_ptr() + (k * P + int(starts[j])) * es
+                                     for k in range(cfg.K) for j in range(len(numel))])
+        xp = gpu.lib.make_ptr_array([hx.data_ptr() + int(starts[j]) * 4 for j in range(len(numel))])
+        for t in range(4):
+            g = _grads(cfg, P, t)
+            hg.copy_(torch.from_numpy(g.view(np.int16) if precision else g))
+            synced = gpu.lib.step_host(gp, cfg.lr, cfg.eta, xp, hb.data_ptr(), gpu.stream)
+            orc.step(g, cfg.lr, cfg.eta)
+            assert synced == ((t + 1) % 2 == 0)
+            assert hb.tolist() == [int(v) for v in orc.last_b]
+            if synced:
+                assert np.array_equal(hx.numpy(), orc.xg)
+        compare_state(gpu.state(), orc, exact=True)
