@@ -1,0 +1,376 @@
+#!/usr/bin/env python
+"""Benchmark of the PALSGD update / synchronisation path.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+A "step" is one iteration of Algorithm 1 for all K workers: the fused inner
+kernel (branch draw + optimizer step or pull), plus the outer-sync kernel on
+every H-th step.  The metric is worker-element updates per second (K*P per
+step), whole job.  Inputs are synthetic (model-shaped buffers, seeded normal
+values) and resident in device memory before the timed region; the `e2e` figure
+repeats the measurement through palsgd_step_host with gradients in pinned host
+memory and results read back to the host every step.
+
+With N > 1 (launched by torch.distributed.run) every rank runs an independent
+replica of the workload on its own GPU: the path has no cross-GPU exchange.
+One JSON line is printed by rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+import workloads as W  # noqa: E402
+
+METRIC = "param_updates_per_s"
+UNIT = "worker-element updates/s"
+DEFAULT_WORKLOAD = "c3_gptneo125m_bf16"
+
+
+# ----------------------------------------------------------------------------- helpers
+
+def measured_peak_gbs():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    except Exception:
+        return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+def inner_bytes_per_element(cfg, pull: bool) -> int:
+    """Algorithmic HBM bytes per worker-element of the fused inner kernel."""
+    bf = cfg.precision == 1
+    if pull:                       # read x, x_g; write x (+ bf16 working copy)
+        return 14 if bf else 12
+    if cfg.inner == 0:             # AdamW: read g, x, m, v; write x, m, v (+ bf16 copy; bf16 g)
+        return 28
+    return 18 if bf else 20        # momentum SGD: read g, x, buf; write x, buf
+
+
+def outer_bytes_per_param(cfg) -> int:
+    """Read K slots, x_g, u; write x_g, u, K slots (+ K bf16 working copies)."""
+    return (10 if cfg.precision == 1 else 8) * cfg.K + 16
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle sampling while the timed region runs."""
+
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.gpu_index)], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()                      # the exact process started above
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, pw, reasons = [], [], [], set()
+        try:
+            for line in open(self.path):
+                f = [x.strip() for x in line.split(",")]
+                if len(f) < 9:
+                    continue
+                try:
+                    sm.append(float(f[1])); mx.append(float(f[2])); pw.append(float(f[3]))
+                except ValueError:
+                    continue
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown",
+                                      "sw_power_cap"), f[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+        finally:
+            try:
+                os.unlink(self.path)
+            except OSError:
+                pass
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(pw) if pw else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ----------------------------------------------------------------------------- CPU oracle leg
+
+def time_oracle(cfg, steps: int, P_sample: int, H: int):
+    """The CPU oracle, as it stands, on the first P_sample elements of the workload."""
+    import oracle
+    K = cfg.K
+    x_init = W.init_params_host(W.flat_shape(P_sample), cfg.param_seed, cfg.init_std)
+    o = oracle.Oracle(np.tile(x_init, (K, 1)), dtype="f32", K=K, H=H, p=cfg.p, inner=cfg.inner,
+                      beta1=cfg.beta1, beta2=cfg.beta2, eps=cfg.eps, weight_decay=cfg.weight_decay,
+                      momentum=cfg.momentum, outer_lr=cfg.outer_lr, outer_momentum=cfg.outer_momentum,
+                      outer_nesterov=cfg.outer_nesterov, seed=cfg.decision_seed, precision=cfg.precision)
+    g = np.stack([W.grads_host(P_sample, cfg.grad_seed, 0, k, cfg.grad_std) for k in range(K)])
+    if cfg.precision == 1:
+        g = W.bf16_bits_from_f32_host(g)
+    o.step(g, cfg.lr, cfg.eta)                     # warm the pages
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        o.step(g, cfg.lr, cfg.eta)
+    dt = time.perf_counter() - t0
+    return K * P_sample * steps / dt, dt, oracle.get_threads(), o.n_outer
+
+
+def run_reference(args, cfg):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    P_sample = min(cfg.P, 1 << 21)
+    H = max(2, min(cfg.H, args.steps))
+    t_all = []
+    for _ in range(max(args.warmup, 0)):
+        time_oracle(cfg, 1, P_sample, H)
+    value, dt, cores, n_outer = time_oracle(cfg, args.steps, P_sample, H)
+    sample = (f"first {P_sample} of {cfg.P} elements per worker, K={cfg.K}, {args.steps} steps, "
+              f"H={H} ({n_outer} outer syncs)")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32" if cfg.precision == 0 else "f32 math, bf16 params/grads",
+        "data": "synthetic", "config": workload_config(cfg, args),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def workload_config(cfg, args) -> dict:
+    return {"workload": cfg.name, "K": cfg.K, "P": cfg.P, "n_tensors": len(cfg.tensors), "H": cfg.H,
+            "p": cfg.p, "eta": cfg.eta, "lr": cfg.lr,
+            "inner": "adamw" if cfg.inner == 0 else "sgdm",
+            "precision": "bf16 params+grads, fp32 master/moments" if cfg.precision == 1 else "fp32",
+            "parallelism": f"replicas x{args.gpus}" if args.gpus > 1 else "single GPU",
+            "l2": "state far larger than L2 (no flush needed)"
+                  if cfg.K * cfg.P * 16 > 4 * 126e6 else "L2-affected: state comparable to the 126 MB L2"}
+
+
+# ----------------------------------------------------------------------------- GPU leg
+
+def run_ours(args, cfg):
+    import torch
+    import torch.distributed as dist
+    import paper_2504_18454_b200 as P
+    from paper_2504_18454_b200.arena import ReplicaArena
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.gpus > 1 and world != args.gpus:
+        raise SystemExit("launch with: python -m torch.distributed.run --nnodes=1 --nproc-per-node N "
+                         "--master-addr 127.0.0.1 --master-port P bench.py --gpus N ...")
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    # CPU baseline first (rank 0, single-GPU runs only), before the GPU is busy
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        P_s = min(cfg.P, 1 << 21)
+        H_s = 64
+        value, dt, cores, n_outer = time_oracle(cfg, 64, P_s, H_s)
+        cpu_baseline = {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                        "sample": f"first {P_s} of {cfg.P} elements per worker, K={cfg.K}, 64 steps incl. "
+                                  f"{n_outer} outer sync, {dt:.1f} s"}
+
+    # ---- buffers: seeded synthetic values, resident in HBM
+    K, Pn = cfg.K, cfg.P
+    numel = [t.numel for t in cfg.tensors]
+    arena = ReplicaArena(numel, K, precision=cfg.precision, inner=cfg.inner, device=dev)
+    x_init = torch.from_numpy(W.init_params_host(cfg.tensors, cfg.param_seed + rank, cfg.init_std)).to(dev)
+    arena.model.copy_(x_init[None].expand(K, Pn))
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(cfg.grad_seed + rank)
+    for k in range(K):
+        arena.rows("grad")[k].copy_(
+            torch.randn(Pn, generator=gen, device=dev, dtype=torch.float32).mul_(cfg.grad_std))
+    del x_init
+    stream = torch.cuda.current_stream(dev).cuda_stream
+    ctx = arena.make_context(
+        stream=stream, H=cfg.H, p=cfg.p, beta1=cfg.beta1, beta2=cfg.beta2, eps=cfg.eps,
+        weight_decay=cfg.weight_decay, momentum=cfg.momentum, outer_lr=cfg.outer_lr,
+        outer_momentum=cfg.outer_momentum, outer_nesterov=cfg.outer_nesterov, seed=cfg.decision_seed)
+
+    t_host = 0                                           # mirrors the library's step counter
+    def one_step(ev_list=None):
+        nonlocal t_host
+        if ev_list is not None:
+            e = torch.cuda.Event(enable_timing=True); e.record(); ev_list.append(("inner", t_host, e))
+        ctx.inner_step(cfg.lr, cfg.eta, stream)
+        t_host += 1
+        if t_host % cfg.H == 0:
+            if ev_list is not None:
+                e = torch.cuda.Event(enable_timing=True); e.record(); ev_list.append(("outer", t_host, e))
+            ctx.outer_sync(stream)
+
+    for _ in range(max(args.warmup, 3)):
+        one_step()
+    # align the timed region so that it contains floor(steps / H) outer syncs in a fixed pattern
+    while t_host % cfg.H != 0:
+        one_step()
+
+    # ---- timed region: device-resident inputs
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    launches0 = ctx.get_launch_count()
+    events = []
+    barrier()
+    e_start = torch.cuda.Event(enable_timing=True); e_end = torch.cuda.Event(enable_timing=True)
+    e_start.record()
+    for _ in range(args.steps):
+        one_step(events)
+    e_end.record()
+    barrier()
+    ms_total = e_start.elapsed_time(e_end)
+    launches = ctx.get_launch_count() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    events.append(("end", t_host, e_end))
+
+    # per-kernel durations (event to next event on the same stream) and algorithmic bytes
+    inner_ms = inner_bytes = outer_ms = outer_bytes = 0.0
+    n_inner = n_outer = 0
+    for (kind, t_after, ev), (_, _, nxt) in zip(events[:-1], events[1:]):
+        d = ev.elapsed_time(nxt)
+        if kind == "inner":
+            b = sum(inner_bytes_per_element(cfg, bool(P.decision(cfg.decision_seed, t_after, k, cfg.p)))
+                    for k in range(K)) * Pn
+            inner_ms += d; inner_bytes += b; n_inner += 1
+        else:
+            outer_ms += d; outer_bytes += outer_bytes_per_param(cfg) * Pn; n_outer += 1
+
+    # ---- end to end: gradients from pinned host memory, results back to the host, every step
+    e2e = None
+    if not args.no_e2e:
+        gdt = torch.bfloat16 if cfg.precision == 1 else torch.float32
+        h_grad = torch.empty((K, Pn), dtype=gdt).pin_memory()
+        h_grad.copy_(arena.rows("grad"))
+        h_glob = torch.empty(Pn, dtype=torch.float32).pin_memory()
+        h_dec = torch.zeros(K, dtype=torch.uint8).pin_memory()
+        es = h_grad.element_size()
+        gp = ctx.make_ptr_array([h_grad.data_ptr() + (k * Pn + arena.starts[j]) * es
+                                 for k in range(K) for j in range(len(numel))])
+        xp = ctx.make_ptr_array([h_glob.data_ptr() + arena.starts[j] * 4 for j in range(len(numel))])
+        e2e_steps = args.e2e_steps if args.e2e_steps > 0 else min(args.steps, cfg.H)
+        for _ in range(2):
+            ctx.step_host(gp, cfg.lr, cfg.eta, xp, h_dec.data_ptr(), stream); t_host += 1
+        while t_host % cfg.H != (cfg.H - e2e_steps) % cfg.H:          # end the region on a sync step
+            ctx.step_host(gp, cfg.lr, cfg.eta, xp, h_dec.data_ptr(), stream); t_host += 1
+        barrier()
+        s0 = torch.cuda.Event(enable_timing=True); s1 = torch.cuda.Event(enable_timing=True)
+        s0.record()
+        syncs = 0
+        for _ in range(e2e_steps):
+            syncs += int(ctx.step_host(gp, cfg.lr, cfg.eta, xp, h_dec.data_ptr(), stream)); t_host += 1
+        s1.record()
+        barrier()
+        ms_e2e = s0.elapsed_time(s1)
+        e2e = {"ms": ms_e2e, "steps": e2e_steps, "syncs": syncs,
+               "h2d": K * Pn * es, "d2h": K + syncs * Pn * 4 / e2e_steps}
+
+    # ---- max over ranks
+    if world > 1:
+        t = torch.tensor([ms_total, e2e["ms"] if e2e else 0.0], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total, ms_e2e_max = float(t[0]), float(t[1])
+        if e2e:
+            e2e["ms"] = ms_e2e_max
+    if rank == 0:
+        peak, peak_src = measured_peak_gbs()
+        value = world * K * Pn * args.steps / (ms_total * 1e-3)
+        inner_gbs = inner_bytes / (inner_ms * 1e-3) / 1e9 if inner_ms else None
+        outer_gbs = outer_bytes / (outer_ms * 1e-3) / 1e9 if outer_ms else None
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_total / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32" if cfg.precision == 0 else "f32 math, bf16 params/grads",
+            "data": "synthetic", "config": workload_config(cfg, args),
+            "roofline": {"bound": "hbm", "kernel": "palsgd_inner_kernel", "achieved": inner_gbs,
+                         "peak": peak, "unit": "GB/s", "frac": inner_gbs / peak if inner_gbs else None,
+                         "traffic": None, "peak_source": peak_src, "frac_of_8000_nominal":
+                         inner_gbs / 8000.0 if inner_gbs else None,
+                         "launches": n_inner, "avg_ms": inner_ms / n_inner if n_inner else None,
+                         "alg_bytes_per_launch": inner_bytes / n_inner if n_inner else None},
+            "roofline_outer": {"bound": "hbm", "kernel": "palsgd_outer_kernel", "achieved": outer_gbs,
+                               "peak": peak, "unit": "GB/s", "frac": outer_gbs / peak if outer_gbs else None,
+                               "traffic": None, "frac_of_8000_nominal": outer_gbs / 8000.0 if outer_gbs else None,
+                               "launches": n_outer, "avg_ms": outer_ms / n_outer if n_outer else None,
+                               "alg_bytes_per_launch": outer_bytes / n_outer if n_outer else None,
+                               "params_per_s": Pn * n_outer / (outer_ms * 1e-3) if outer_ms else None},
+            "cpu_baseline": cpu_baseline,
+            "e2e": ({"value": world * K * Pn * e2e["steps"] / (e2e["ms"] * 1e-3), "unit": UNIT,
+                     "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
+                     "steps": e2e["steps"], "outer_syncs": e2e["syncs"]} if e2e else None),
+            "gpu_launches": launches,
+            "clocks": clocks,
+        }
+        print(json.dumps(line), flush=True)
+    ctx.destroy()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=256)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(W.CONFIGS))
+    ap.add_argument("--e2e-steps", type=int, default=0, help="0 = min(steps, H)")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    cfg = W.get_config(args.workload)
+    if args.impl == "reference":
+        if args.steps == 256:
+            args.steps = 32                       # a bounded sample: keep the CPU run to about a minute
+        run_reference(args, cfg)
+    else:
+        run_ours(args, cfg)
+
+
+if __name__ == "__main__":
+    main()

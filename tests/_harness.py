@@ -11,7 +11,7 @@ import oracle
 import paper_2504_18454_b200 as P
 
 GUARD = 64                  # sentinel elements on both sides of every arena row
-SENTINEL = 1234.5
+SENTINEL = 1536.0            # exactly representable in bf16 too
 REL_TOL, ABS_FLOOR = 1e-6, 1e-7   # fp32 state: max |rel err| <= 1e-6 with abs floor 1e-7
 
 

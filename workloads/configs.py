@@ -73,6 +73,13 @@ CONFIGS: Dict[str, WorkloadConfig] = {
     "c3_gptneo125m_bf16": WorkloadConfig(
         name="c3_gptneo125m_bf16", shape=gptneo_125m_shape,
         K=8, H=128, p=0.1, eta=16.0, lr=1e-3, T=512, precision=BF16_MASTER),
+    # profiling-sized stand-ins (a few GB, larger than L2) for ncu captures of the same kernels
+    "prof_flat16m_bf16": WorkloadConfig(
+        name="prof_flat16m_bf16", shape=lambda: flat_shape(1 << 24),
+        K=8, H=8, p=0.1, eta=16.0, lr=1e-3, T=16, precision=BF16_MASTER),
+    "prof_flat16m_fp32": WorkloadConfig(
+        name="prof_flat16m_fp32", shape=lambda: flat_shape(1 << 24),
+        K=8, H=8, p=0.1, eta=16.0, lr=1e-3, T=16),
 }
 
 
