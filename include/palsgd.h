@@ -180,10 +180,12 @@ int palsgd_set_counters(palsgd_ctx* ctx, uint64_t t, const uint64_t* s_k, uint64
 /* Number of kernels this context has launched so far (host-side count). */
 int palsgd_get_launch_count(palsgd_ctx* ctx, uint64_t* n_launches);
 
-/* Launch-shape knobs (advanced; results never depend on them).  value = the
- * largest grid a launch may use, CTAs looping over work items beyond it;
- * 0 (default) = one CTA per work item. */
-enum { PALSGD_TUNE_INNER_GRID_CAP = 0, PALSGD_TUNE_OUTER_GRID_CAP = 1 };
+/* Launch-shape knobs (advanced; results never depend on them).
+ * *_GRID_CAP: the largest grid a launch may use, CTAs looping over work items
+ * beyond it; 0 (default) = one CTA per work item.
+ * INNER_VARIANT: which compiled shape of the fused inner kernel runs (loads in
+ * flight per thread x CTAs per SM); 0 = the library's default, unknown = default. */
+enum { PALSGD_TUNE_INNER_GRID_CAP = 0, PALSGD_TUNE_OUTER_GRID_CAP = 1, PALSGD_TUNE_INNER_VARIANT = 2 };
 int palsgd_set_tuning(palsgd_ctx* ctx, int knob, int64_t value);
 
 /* The branch draw as a pure host function: 1 = pseudo-sync, 0 = gradient step;

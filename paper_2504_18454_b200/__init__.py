@@ -17,4 +17,5 @@ from .binding import (  # noqa: F401
     PREC_BF16_MASTER,
     TUNE_INNER_GRID_CAP,
     TUNE_OUTER_GRID_CAP,
+    TUNE_INNER_VARIANT,
 )

@@ -40,6 +40,7 @@ struct palsgd_ctx {
     uint64_t t = 0, n_outer = 0, launches = 0;
     uint64_t thr = 0;
     int grid_cap_inner = 0, grid_cap_outer = 0;   // 0 = one CTA per work item
+    int inner_variant = 0;                        // launch shape of the inner kernel, 0 = default
     std::string cuda_err;
 };
 
@@ -125,6 +126,25 @@ OuterArgs outer_args(const palsgd_ctx* ctx)
     return a;
 }
 
+// Launch shapes of the fused inner kernel: U = 128-bit loads in flight per
+// stream and thread, MINB = CTAs per SM the register budget is held to.
+template <int INNER, int PREC>
+void launch_inner_variant(int variant, unsigned grid, cudaStream_t s, const InnerArgs& a)
+{
+    switch (variant) {
+        case 1:  palsgd_inner_kernel<INNER, PREC, 1, 4><<<grid, kThreads, 0, s>>>(a); break;
+        case 2:  palsgd_inner_kernel<INNER, PREC, 1, 3><<<grid, kThreads, 0, s>>>(a); break;
+        case 3:  palsgd_inner_kernel<INNER, PREC, 2, 2><<<grid, kThreads, 0, s>>>(a); break;
+        case 4:  palsgd_inner_kernel<INNER, PREC, 2, 3><<<grid, kThreads, 0, s>>>(a); break;
+        case 5:  palsgd_inner_kernel<INNER, PREC, 4, 1><<<grid, kThreads, 0, s>>>(a); break;
+        case 6:  palsgd_inner_kernel<INNER, PREC, 1, 6><<<grid, kThreads, 0, s>>>(a); break;
+        default:      // measured best on B200: one 128-bit load per stream and thread, many CTAs per SM
+            if (PREC) palsgd_inner_kernel<INNER, PREC, 1, 4><<<grid, kThreads, 0, s>>>(a);
+            else      palsgd_inner_kernel<INNER, PREC, 1, 6><<<grid, kThreads, 0, s>>>(a);
+            break;
+    }
+}
+
 int launch_inner(palsgd_ctx* ctx, const InnerArgs& a, cudaStream_t s)
 {
     const uint64_t n_items = (uint64_t)ctx->tb.n_chunks * ctx->cfg.K;
@@ -132,11 +152,12 @@ int launch_inner(palsgd_ctx* ctx, const InnerArgs& a, cudaStream_t s)
     const unsigned grid = grid_for(n_items, ctx->grid_cap_inner);
     const bool adam = ctx->cfg.inner == PALSGD_INNER_ADAMW;
     const bool bf = ctx->cfg.precision == PALSGD_PREC_BF16_MASTER;
+    const int v = ctx->inner_variant;
     return launch_checked(ctx, [&] {
-        if (adam && !bf)      palsgd_inner_kernel<0, 0, 4><<<grid, kThreads, 0, s>>>(a);
-        else if (!adam && !bf) palsgd_inner_kernel<1, 0, 4><<<grid, kThreads, 0, s>>>(a);
-        else if (adam && bf)  palsgd_inner_kernel<0, 1, 2><<<grid, kThreads, 0, s>>>(a);
-        else                  palsgd_inner_kernel<1, 1, 2><<<grid, kThreads, 0, s>>>(a);
+        if (adam && !bf)       launch_inner_variant<0, 0>(v, grid, s, a);
+        else if (!adam && !bf) launch_inner_variant<1, 0>(v, grid, s, a);
+        else if (adam && bf)   launch_inner_variant<0, 1>(v, grid, s, a);
+        else                   launch_inner_variant<1, 1>(v, grid, s, a);
     });
 }
 
@@ -501,6 +522,7 @@ extern "C" int palsgd_set_tuning(palsgd_ctx* ctx, int knob, int64_t value)
     switch (knob) {
         case PALSGD_TUNE_INNER_GRID_CAP: ctx->grid_cap_inner = (int)value; return PALSGD_OK;
         case PALSGD_TUNE_OUTER_GRID_CAP: ctx->grid_cap_outer = (int)value; return PALSGD_OK;
+        case PALSGD_TUNE_INNER_VARIANT:  ctx->inner_variant = (int)value; return PALSGD_OK;
         default: return PALSGD_EINVAL;
     }
 }

@@ -366,8 +366,8 @@ __device__ __forceinline__ void grad_item(const Tables& tb, uint32_t k, const Ch
 // Every CTA recomputes the K decisions of step t from the counter-based
 // stream; the last CTA to finish advances the device counters.
 
-template <int INNER, int PREC, int U>
-__global__ void __launch_bounds__(kThreads)
+template <int INNER, int PREC, int U, int MINB>
+__global__ void __launch_bounds__(kThreads, MINB)
 palsgd_inner_kernel(const __grid_constant__ InnerArgs a)
 {
     __shared__ unsigned char s_pull[kMaxWorkers];
