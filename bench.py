@@ -232,6 +232,8 @@ def run_ours(args, cfg):
         weight_decay=cfg.weight_decay, momentum=cfg.momentum, outer_lr=cfg.outer_lr,
         outer_momentum=cfg.outer_momentum, outer_nesterov=cfg.outer_nesterov, seed=cfg.decision_seed)
 
+    if args.inner_variant:
+        ctx.set_tuning(P.TUNE_INNER_VARIANT, args.inner_variant)
     t_host = 0                                           # mirrors the library's step counter
     def one_step(ev_list=None):
         nonlocal t_host
@@ -360,6 +362,7 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(W.CONFIGS))
     ap.add_argument("--e2e-steps", type=int, default=0, help="0 = min(steps, H)")
+    ap.add_argument("--inner-variant", type=int, default=0, help="palsgd_set_tuning(INNER_VARIANT); 0 = default")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

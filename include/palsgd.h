@@ -55,7 +55,8 @@ typedef enum palsgd_status {
     PALSGD_ECUDA        = -3,   /* a CUDA runtime call or a kernel launch failed                     */
     PALSGD_ESTATE       = -4,   /* call not valid in this state (e.g. undefined coefficient)         */
     PALSGD_ENOMEM       = -5,   /* host or device allocation failed                                  */
-    PALSGD_EUNSUPPORTED = -6    /* combination not built                                             */
+    PALSGD_EUNSUPPORTED = -6,   /* combination not built                                             */
+    PALSGD_ETIMEOUT     = -7    /* a bounded wait inside a kernel expired (reported by get_counters)  */
 } palsgd_status;
 
 enum { PALSGD_INNER_ADAMW = 0, PALSGD_INNER_SGDM = 1 };
@@ -167,7 +168,8 @@ int palsgd_step_host(palsgd_ctx* ctx, const void* const* h_grad, double lr_t, do
  * Read the counters (SYNCHRONISES the stream): t = completed steps, s_k[K] =
  * gradient steps taken by worker k, n_outer = outer syncs, last_b[K] = decisions
  * of the latest inner step.  Any output pointer may be NULL.
- * Errors: ESTATE if the device-side t disagrees with the host mirror; ECUDA.
+ * Errors: ETIMEOUT if a kernel recorded an expired wait; ESTATE if the device-side
+ * t disagrees with the host mirror; ECUDA.
  */
 int palsgd_get_counters(palsgd_ctx* ctx, uint64_t* t, uint64_t* s_k, uint64_t* n_outer,
                         uint8_t* last_b, void* stream);
@@ -183,9 +185,20 @@ int palsgd_get_launch_count(palsgd_ctx* ctx, uint64_t* n_launches);
 /* Launch-shape knobs (advanced; results never depend on them).
  * *_GRID_CAP: the largest grid a launch may use, CTAs looping over work items
  * beyond it; 0 (default) = one CTA per work item.
- * INNER_VARIANT: which compiled shape of the fused inner kernel runs (loads in
- * flight per thread x CTAs per SM); 0 = the library's default, unknown = default. */
-enum { PALSGD_TUNE_INNER_GRID_CAP = 0, PALSGD_TUNE_OUTER_GRID_CAP = 1, PALSGD_TUNE_INNER_VARIANT = 2 };
+ * INNER_VARIANT: which compiled form of the fused inner kernel runs: 1..9 =
+ * register-path shapes (loads in flight per thread x CTAs per SM), 10 / 11 / 12 = the
+ * persistent shared-memory-ring form with 512 / 256 / 1024 consumer threads; 0 = the
+ * library's default, unknown = default.
+ * PIPE_STAGES: ring depth of the persistent form; 0 = as many as fit.
+ * CHUNK_MAJOR: order of the (chunk, worker) work items of the register-path inner
+ * kernel: 0 = worker index fastest (default), 1 = chunk index fastest.
+ * OUTER_SUB_ELEMS: elements per work item of the outer kernel (a slice of a chunk),
+ * a multiple of 1024; default 1024.
+ * (Environment variable PALSGD_CHUNK_ELEMS, read by palsgd_init: elements per chunk
+ * = per work item of the inner kernel, a multiple of 1024; default 4096 for fp32 AdamW,
+ * 8192 otherwise.) */
+enum { PALSGD_TUNE_INNER_GRID_CAP = 0, PALSGD_TUNE_OUTER_GRID_CAP = 1, PALSGD_TUNE_INNER_VARIANT = 2,
+       PALSGD_TUNE_PIPE_STAGES = 3, PALSGD_TUNE_CHUNK_MAJOR = 4, PALSGD_TUNE_OUTER_SUB_ELEMS = 5 };
 int palsgd_set_tuning(palsgd_ctx* ctx, int knob, int64_t value);
 
 /* The branch draw as a pure host function: 1 = pseudo-sync, 0 = gradient step;

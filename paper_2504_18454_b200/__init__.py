@@ -18,4 +18,5 @@ from .binding import (  # noqa: F401
     TUNE_INNER_GRID_CAP,
     TUNE_OUTER_GRID_CAP,
     TUNE_INNER_VARIANT,
+    TUNE_PIPE_STAGES,
 )

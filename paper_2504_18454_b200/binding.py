@@ -10,7 +10,7 @@ LIB_PATH = HERE / "libpalsgd.so"
 
 INNER_ADAMW, INNER_SGDM = 0, 1
 PREC_FP32, PREC_BF16_MASTER = 0, 1
-TUNE_INNER_GRID_CAP, TUNE_OUTER_GRID_CAP, TUNE_INNER_VARIANT = 0, 1, 2
+TUNE_INNER_GRID_CAP, TUNE_OUTER_GRID_CAP, TUNE_INNER_VARIANT, TUNE_PIPE_STAGES = 0, 1, 2, 3
 MAX_WORKERS = 64
 
 

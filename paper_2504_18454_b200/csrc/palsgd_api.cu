@@ -7,14 +7,17 @@
 // n_outer for the "(t+1) mod H" test.
 #include "../../include/palsgd.h"
 
+#include <algorithm>
 #include <cmath>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <string>
 #include <vector>
 
 #include "palsgd_kernels.cuh"
+#include "palsgd_pipe.cuh"
 
 using namespace palsgd;
 
@@ -41,6 +44,11 @@ struct palsgd_ctx {
     uint64_t thr = 0;
     int grid_cap_inner = 0, grid_cap_outer = 0;   // 0 = one CTA per work item
     int inner_variant = 0;                        // launch shape of the inner kernel, 0 = default
+    int pipe_stages = 0;                          // ring depth of the pipelined kernel, 0 = as many as fit
+    int chunk_major = 0;                          // work-item order of the register-path inner kernel
+    uint32_t chunk_elems = kChunkElems;           // elements per chunk-table entry (fixed at init)
+    uint32_t outer_sub_elems = kOuterSubElems;    // elements per work item of the outer kernel
+    int sm_count = 0, smem_optin = 0;             // device attributes read at init
     std::string cuda_err;
 };
 
@@ -123,6 +131,8 @@ OuterArgs outer_args(const palsgd_ctx* ctx)
     a.lr = (float)ctx->cfg.outer_lr;
     a.Kf = (float)ctx->cfg.K;
     a.nesterov = ctx->cfg.outer_nesterov;
+    a.sub_elems = ctx->outer_sub_elems;
+    a.parts = (ctx->chunk_elems + a.sub_elems - 1) / a.sub_elems;
     return a;
 }
 
@@ -138,6 +148,12 @@ void launch_inner_variant(int variant, unsigned grid, cudaStream_t s, const Inne
         case 4:  palsgd_inner_kernel<INNER, PREC, 2, 3><<<grid, kThreads, 0, s>>>(a); break;
         case 5:  palsgd_inner_kernel<INNER, PREC, 4, 1><<<grid, kThreads, 0, s>>>(a); break;
         case 6:  palsgd_inner_kernel<INNER, PREC, 1, 6><<<grid, kThreads, 0, s>>>(a); break;
+        case 7:  palsgd_inner_kernel<INNER, PREC, 0, 6><<<grid, kThreads, 0, s>>>(a); break;
+        case 8:  palsgd_inner_kernel<INNER, PREC, 0, 5><<<grid, kThreads, 0, s>>>(a); break;
+        case 9:  palsgd_inner_kernel<INNER, PREC, 0, 8><<<grid, kThreads, 0, s>>>(a); break;
+        case 13: palsgd_inner_kernel<INNER, PREC, -1, 4><<<grid, kThreads, 0, s>>>(a); break;
+        case 14: palsgd_inner_kernel<INNER, PREC, -1, 3><<<grid, kThreads, 0, s>>>(a); break;
+        case 15: palsgd_inner_kernel<INNER, PREC, -1, 5><<<grid, kThreads, 0, s>>>(a); break;
         default:      // measured best on B200: one 128-bit load per stream and thread, many CTAs per SM
             if (PREC) palsgd_inner_kernel<INNER, PREC, 1, 4><<<grid, kThreads, 0, s>>>(a);
             else      palsgd_inner_kernel<INNER, PREC, 1, 6><<<grid, kThreads, 0, s>>>(a);
@@ -145,8 +161,60 @@ void launch_inner_variant(int variant, unsigned grid, cudaStream_t s, const Inne
     }
 }
 
+using PipeKernel = void (*)(const InnerArgs, uint32_t, uint32_t);
+template <int INNER, int PREC, int NC>
+PipeKernel pipe_kernel_ptr()
+{
+    if constexpr (NC == 0) return palsgd_inner_pipe_all_kernel<INNER, PREC>;
+    else return palsgd_inner_pipe_kernel<INNER, PREC, NC>;
+}
+
+// Persistent TMA-ring kernel: one CTA per SM, as many stages as shared memory holds.
+template <int INNER, int PREC, int NC>
+int launch_inner_pipe(palsgd_ctx* ctx, const InnerArgs& a, cudaStream_t s)
+{
+    constexpr uint32_t stage_bytes = ((INNER == 0 ? 12u : 8u) + (PREC ? 2u : 4u)) * kStageElems;
+    const int budget = ctx->smem_optin - 4096;              // static shared memory and the system's share
+    int stages = std::min<int>(kPipeMaxStages, budget / (int)stage_bytes);
+    if (ctx->pipe_stages > 0) stages = std::min(stages, ctx->pipe_stages);
+    if (stages < 2) return PALSGD_EUNSUPPORTED;
+    const size_t dyn = (size_t)stages * stage_bytes;
+    auto kernel = pipe_kernel_ptr<INNER, PREC, NC>();
+    constexpr unsigned threads = NC == 0 ? 1024u : (unsigned)NC + 32u;
+    static int attr_for_device = -1;                         // opt in to large dynamic shared memory once
+    int dev = 0;
+    PALSGD_CUDA(ctx, cudaGetDevice(&dev));
+    if (attr_for_device != dev) {
+        PALSGD_CUDA(ctx, cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, budget));
+        attr_for_device = dev;
+    }
+    const uint64_t n_items = (uint64_t)ctx->tb.n_full * ctx->cfg.K * (ctx->chunk_elems / kStageElems);
+    const int cap = ctx->grid_cap_inner > 0 ? ctx->grid_cap_inner : ctx->sm_count;
+    const unsigned grid = grid_for(n_items, cap);
+    return launch_checked(ctx, [&] { kernel<<<grid, threads, dyn, s>>>(a, (uint32_t)stages, stage_bytes); });
+}
+
+// NC = 0 selects the form in which all 1024 threads consume and thread 0 also produces.
+template <int INNER, int PREC>
+int launch_inner_pipe_nc(palsgd_ctx* ctx, int variant, const InnerArgs& a, cudaStream_t s)
+{
+    if (variant == 11) return launch_inner_pipe<INNER, PREC, 256>(ctx, a, s);
+    if (variant == 10) return launch_inner_pipe<INNER, PREC, 512>(ctx, a, s);
+    return launch_inner_pipe<INNER, PREC, 0>(ctx, a, s);
+}
+
 int launch_inner(palsgd_ctx* ctx, const InnerArgs& a, cudaStream_t s)
 {
+    if (ctx->inner_variant >= 10 && ctx->inner_variant <= 12 && ctx->tb.n_full > 0 &&
+        ctx->chunk_elems % kStageElems == 0) {
+        const bool adam_ = ctx->cfg.inner == PALSGD_INNER_ADAMW;
+        const bool bf_ = ctx->cfg.precision == PALSGD_PREC_BF16_MASTER;
+        const int v_ = ctx->inner_variant;
+        if (adam_ && !bf_)  return launch_inner_pipe_nc<0, 0>(ctx, v_, a, s);
+        if (!adam_ && !bf_) return launch_inner_pipe_nc<1, 0>(ctx, v_, a, s);
+        if (adam_ && bf_)   return launch_inner_pipe_nc<0, 1>(ctx, v_, a, s);
+        return launch_inner_pipe_nc<1, 1>(ctx, v_, a, s);
+    }
     const uint64_t n_items = (uint64_t)ctx->tb.n_chunks * ctx->cfg.K;
     // with nothing to stream a one-CTA launch still advances the counters
     const unsigned grid = grid_for(n_items, ctx->grid_cap_inner);
@@ -241,6 +309,12 @@ extern "C" int palsgd_init(palsgd_ctx** out, const palsgd_config* cfg, size_t n_
     const size_t n_seg = ctx->segs.size();
 
     // ---- chunk table and per-segment vector-path flag
+    // Elements per inner work item, measured best on B200: 4096 for fp32 AdamW, 8192 otherwise.
+    ctx->chunk_elems = (!bf && adam) ? 4096u : kChunkElems;
+    if (const char* e = std::getenv("PALSGD_CHUNK_ELEMS")) {      // tuning aid: a multiple of 1024
+        const long v = std::atol(e);
+        if (v >= 1024 && v <= (1 << 20) && v % 1024 == 0) ctx->chunk_elems = (uint32_t)v;
+    }
     std::vector<Chunk> chunks;
     for (size_t s = 0; s < n_seg; ++s) {
         const Segment& sg = ctx->segs[s];
@@ -249,12 +323,16 @@ extern "C" int palsgd_init(palsgd_ctx** out, const palsgd_config* cfg, size_t n_
             for (const Kind& kd : kinds)
                 if (kd.present && !aligned(buf_ptr(bufs, kd.id, (size_t)k * n_tensors + sg.first_tensor), 16))
                     vec = false;
-        for (uint64_t off = 0; off < sg.numel; off += kChunkElems) {
-            const uint64_t len = sg.numel - off < kChunkElems ? sg.numel - off : kChunkElems;
+        for (uint64_t off = 0; off < sg.numel; off += ctx->chunk_elems) {
+            const uint64_t len = sg.numel - off < ctx->chunk_elems ? sg.numel - off : ctx->chunk_elems;
             chunks.push_back(Chunk{off, (uint32_t)len, (uint32_t)s | (vec ? kSegVecFlag : 0u)});
         }
     }
     if (chunks.size() > 0x7FFFFFFFull / K) { delete ctx; return PALSGD_EUNSUPPORTED; }
+    // full, aligned chunks first: the pipelined kernel streams exactly those through shared memory
+    const uint32_t full_len = ctx->chunk_elems;
+    auto is_full = [full_len](const Chunk& c) { return (c.seg & kSegVecFlag) && c.len == full_len; };
+    const size_t n_full = std::stable_partition(chunks.begin(), chunks.end(), is_full) - chunks.begin();
 
     // ---- one device blob: [DevState][chunks][7 pointer tables]
     const size_t per_slot = (size_t)K * n_seg * sizeof(void*);
@@ -270,6 +348,14 @@ extern "C" int palsgd_init(palsgd_ctx** out, const palsgd_config* cfg, size_t n_
     if (!chunks.empty()) std::memcpy(host.data() + off_chunks, chunks.data(), chunks.size() * sizeof(Chunk));
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    {
+        int dev = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess) {
+            cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, dev);
+            cudaDeviceGetAttribute(&ctx->smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+        }
+        (void)cudaGetLastError();
+    }
     if (cudaMalloc(&ctx->d_blob, total) != cudaSuccess) {
         cudaError_t e = cudaGetLastError();
         g_noctx_err = std::string("cudaMalloc: ") + cudaGetErrorString(e);
@@ -301,6 +387,8 @@ extern "C" int palsgd_init(palsgd_ctx** out, const palsgd_config* cfg, size_t n_
     tb.n_chunks = (uint32_t)chunks.size();
     tb.n_seg = (uint32_t)n_seg;
     tb.K = K;
+    tb.n_full = (uint32_t)n_full;
+    tb.chunk_elems = ctx->chunk_elems;
     void* t_param = fill_slot_table(0);
     tb.grad = static_cast<const void* const*>(fill_slot_table(1));
     void* t_master = bf ? fill_slot_table(2) : nullptr;
@@ -353,6 +441,7 @@ extern "C" int palsgd_inner_step(palsgd_ctx* ctx, double lr_t, double eta_t, voi
     a.decay = (float)(1.0 - lr_d * c.weight_decay);
     a.mu = (float)c.momentum;
     a.wd = (float)c.weight_decay;
+    a.chunk_major = (uint32_t)ctx->chunk_major;
     int rc = launch_inner(ctx, a, static_cast<cudaStream_t>(stream));
     if (rc) return rc;
     ctx->t += 1;
@@ -383,7 +472,7 @@ extern "C" int palsgd_outer_sync(palsgd_ctx* ctx, void* stream)
     if (!ctx) return PALSGD_EINVAL;
     if (ctx->tb.n_chunks > 0) {
         const OuterArgs a = outer_args(ctx);
-        const unsigned grid = grid_for(ctx->tb.n_chunks, ctx->grid_cap_outer);
+        const unsigned grid = grid_for((uint64_t)ctx->tb.n_chunks * a.parts, ctx->grid_cap_outer);
         cudaStream_t s = static_cast<cudaStream_t>(stream);
         const bool bf = ctx->cfg.precision == PALSGD_PREC_BF16_MASTER;
         int rc = launch_checked(ctx, [&] {
@@ -479,6 +568,7 @@ extern "C" int palsgd_get_counters(palsgd_ctx* ctx, uint64_t* t, uint64_t* s_k, 
         if (s_k) s_k[k] = hs.s[k];
         if (last_b) last_b[k] = hs.last_b[k];
     }
+    if (hs.error != 0) return PALSGD_ETIMEOUT;
     return hs.t == ctx->t ? PALSGD_OK : PALSGD_ESTATE;
 }
 
@@ -523,6 +613,12 @@ extern "C" int palsgd_set_tuning(palsgd_ctx* ctx, int knob, int64_t value)
         case PALSGD_TUNE_INNER_GRID_CAP: ctx->grid_cap_inner = (int)value; return PALSGD_OK;
         case PALSGD_TUNE_OUTER_GRID_CAP: ctx->grid_cap_outer = (int)value; return PALSGD_OK;
         case PALSGD_TUNE_INNER_VARIANT:  ctx->inner_variant = (int)value; return PALSGD_OK;
+        case PALSGD_TUNE_PIPE_STAGES:    ctx->pipe_stages = (int)value; return PALSGD_OK;
+        case PALSGD_TUNE_CHUNK_MAJOR:    ctx->chunk_major = value != 0; return PALSGD_OK;
+        case PALSGD_TUNE_OUTER_SUB_ELEMS:
+            if (value < 1024 || value % 1024 != 0) return PALSGD_EINVAL;
+            ctx->outer_sub_elems = (uint32_t)value;
+            return PALSGD_OK;
         default: return PALSGD_EINVAL;
     }
 }
@@ -545,6 +641,7 @@ extern "C" const char* palsgd_strerror(int status)
         case PALSGD_ESTATE: return "call not valid in this state";
         case PALSGD_ENOMEM: return "out of memory";
         case PALSGD_EUNSUPPORTED: return "unsupported combination";
+        case PALSGD_ETIMEOUT: return "a bounded device-side wait expired";
         default: return "unknown status";
     }
 }

@@ -8,7 +8,11 @@ namespace palsgd {
 
 constexpr uint32_t kMaxWorkers  = 64;      // K <= 64 (worker masks are 64-bit)
 constexpr uint32_t kThreads     = 256;     // threads per CTA of every kernel here
-constexpr uint32_t kChunkElems  = 4096;    // elements per work item (one slot, one chunk)
+constexpr uint32_t kChunkElems  = 8192;    // default elements per chunk-table entry = one work item of the
+                                           // inner kernel (large: amortises the per-CTA prologue and tick)
+constexpr uint32_t kStageElems  = 4096;    // stage size of the shared-memory-ring kernels
+constexpr uint32_t kOuterSubElems = 1024;  // default work item of the outer kernel: a slice of a chunk (small:
+                                           // K+2 streams per element need many CTAs in flight)
 constexpr uint32_t kSegVecFlag  = 0x80000000u;   // Chunk::seg bit: 16-byte vector path allowed
 
 // One work unit of the multi-tensor launch: `len` consecutive elements of
@@ -29,7 +33,7 @@ struct DevState {
     double             pow1[kMaxWorkers];    // beta1^s_k  (running product, binary64)
     double             pow2[kMaxWorkers];    // beta2^s_k
     unsigned int       done;                 // CTAs that finished the current inner launch
-    unsigned int       pad_;
+    unsigned int       error;                // 0, or the code of a bounded wait that expired
     unsigned char      last_b[kMaxWorkers];  // decisions of the latest inner step
 };
 
@@ -39,6 +43,8 @@ struct Tables {
     uint32_t            n_chunks;
     uint32_t            n_seg;
     uint32_t            K;
+    uint32_t            n_full;     // the first n_full chunks are full-size and 16-byte aligned
+    uint32_t            chunk_elems; // elements of a full chunk
     uint32_t            pad_;
     float* const*       xf;         // fp32 model of slot k: params (FP32) or master (BF16_MASTER)
     __nv_bfloat16* const* xw;       // bf16 working params (BF16_MASTER) else nullptr
@@ -59,6 +65,7 @@ struct InnerArgs {
     float    beta_pull;    // fl32(alpha_t * eta_t / p)
     float    b1, b2, omb1, omb2, eps, decay;   // AdamW scalars, each rounded once from binary64
     float    mu, wd;       // momentum SGD scalars
+    uint32_t chunk_major;  // 0: worker index fastest over work items; 1: chunk index fastest
 };
 
 struct PullArgs {
@@ -71,6 +78,8 @@ struct OuterArgs {
     Tables tb;
     float  mu, lr, Kf;
     int    nesterov;
+    uint32_t sub_elems;    // elements per work item (a multiple of 4 * kThreads)
+    uint32_t parts;        // work items per chunk = ceil(chunk_elems / sub_elems)
 };
 
 }  // namespace palsgd

@@ -67,8 +67,8 @@ __device__ __forceinline__ float  compv(const float4& a, int c) { return c == 0 
 // ---------------------------------------------------------------- fp32 chunk bodies
 
 // U independent 128-bit loads per stream are issued before any arithmetic.
-template <int U>
-__device__ __forceinline__ void adamw_chunk_f32(const float* __restrict__ g, float* __restrict__ x,
+template <int U, int NT>
+__device__ __forceinline__ void adamw_chunk_f32(uint32_t tid, const float* __restrict__ g, float* __restrict__ x,
                                                 float* __restrict__ m, float* __restrict__ v,
                                                 uint32_t len, const AdamScalars& s)
 {
@@ -77,82 +77,139 @@ __device__ __forceinline__ void adamw_chunk_f32(const float* __restrict__ g, flo
     float4* x4 = reinterpret_cast<float4*>(x);
     float4* m4 = reinterpret_cast<float4*>(m);
     float4* v4 = reinterpret_cast<float4*>(v);
-    for (uint32_t base = 0; base < n4; base += kThreads * U) {
+    for (uint32_t base = 0; base < n4; base += NT * U) {
         float4 G[U], X[U], M[U], V[U];
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-            const uint32_t i = base + u * kThreads + threadIdx.x;
+            const uint32_t i = base + u * NT + tid;
             if (i < n4) { G[u] = ld_stream(g4 + i); X[u] = ld_stream(x4 + i);
                           M[u] = ld_stream(m4 + i); V[u] = ld_stream(v4 + i); }
         }
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-            const uint32_t i = base + u * kThreads + threadIdx.x;
+            const uint32_t i = base + u * NT + tid;
             if (i < n4) {
                 PALSGD_FOR4(adamw_elem(compv(G[u], c), comp(X[u], c), comp(M[u], c), comp(V[u], c), s))
                 st_stream(x4 + i, X[u]); st_stream(m4 + i, M[u]); st_stream(v4 + i, V[u]);
             }
         }
     }
-    const uint32_t i = (n4 << 2) + threadIdx.x;
+    const uint32_t i = (n4 << 2) + tid;
     if (i < len) { float xi = x[i], mi = m[i], vi = v[i]; adamw_elem(g[i], xi, mi, vi, s);
                    x[i] = xi; m[i] = mi; v[i] = vi; }
 }
 
-template <int U>
-__device__ __forceinline__ void sgdm_chunk_f32(const float* __restrict__ g, float* __restrict__ x,
+template <int U, int NT>
+__device__ __forceinline__ void sgdm_chunk_f32(uint32_t tid, const float* __restrict__ g, float* __restrict__ x,
                                                float* __restrict__ buf, uint32_t len, const SgdScalars& s)
 {
     const uint32_t n4 = len >> 2;
     const float4* g4 = reinterpret_cast<const float4*>(g);
     float4* x4 = reinterpret_cast<float4*>(x);
     float4* b4 = reinterpret_cast<float4*>(buf);
-    for (uint32_t base = 0; base < n4; base += kThreads * U) {
+    for (uint32_t base = 0; base < n4; base += NT * U) {
         float4 G[U], X[U], B[U];
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-            const uint32_t i = base + u * kThreads + threadIdx.x;
+            const uint32_t i = base + u * NT + tid;
             if (i < n4) { G[u] = ld_stream(g4 + i); X[u] = ld_stream(x4 + i); B[u] = ld_stream(b4 + i); }
         }
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-            const uint32_t i = base + u * kThreads + threadIdx.x;
+            const uint32_t i = base + u * NT + tid;
             if (i < n4) {
                 PALSGD_FOR4(sgdm_elem(compv(G[u], c), comp(X[u], c), comp(B[u], c), s))
                 st_stream(x4 + i, X[u]); st_stream(b4 + i, B[u]);
             }
         }
     }
-    const uint32_t i = (n4 << 2) + threadIdx.x;
+    const uint32_t i = (n4 << 2) + tid;
     if (i < len) { float xi = x[i], bi = buf[i]; sgdm_elem(g[i], xi, bi, s); x[i] = xi; buf[i] = bi; }
 }
 
 // x_g is read with the default policy: slots that pull in the same step share it through L2.
-template <int U>
-__device__ __forceinline__ void pull_chunk_f32(float* __restrict__ x, const float* __restrict__ xg,
+template <int U, int NT>
+__device__ __forceinline__ void pull_chunk_f32(uint32_t tid, float* __restrict__ x, const float* __restrict__ xg,
                                                uint32_t len, float beta)
 {
     const uint32_t n4 = len >> 2;
     float4* x4 = reinterpret_cast<float4*>(x);
     const float4* q4 = reinterpret_cast<const float4*>(xg);
-    for (uint32_t base = 0; base < n4; base += kThreads * U) {
+    for (uint32_t base = 0; base < n4; base += NT * U) {
         float4 X[U], Q[U];
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-            const uint32_t i = base + u * kThreads + threadIdx.x;
+            const uint32_t i = base + u * NT + tid;
             if (i < n4) { X[u] = ld_stream(x4 + i); Q[u] = __ldg(q4 + i); }
         }
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-            const uint32_t i = base + u * kThreads + threadIdx.x;
+            const uint32_t i = base + u * NT + tid;
             if (i < n4) {
                 PALSGD_FOR4(comp(X[u], c) = pull_elem(compv(X[u], c), compv(Q[u], c), beta))
                 st_stream(x4 + i, X[u]);
             }
         }
     }
-    const uint32_t i = (n4 << 2) + threadIdx.x;
+    const uint32_t i = (n4 << 2) + tid;
     if (i < len) x[i] = pull_elem(x[i], xg[i], beta);
+}
+
+
+// ---- fp32 bodies with two ADJACENT 128-bit accesses per stream and thread (8 elements, whole
+// 32-byte sectors per thread).  Selected with U = -1 in grad_item / pull_item.
+template <int INNER, int NT>
+__device__ __forceinline__ void grad_chunk_f32_pair(uint32_t tid, const float* __restrict__ g, float* __restrict__ x,
+                                                    float* __restrict__ m, float* __restrict__ v, uint32_t len,
+                                                    const AdamScalars& as, const SgdScalars& ss)
+{
+    const uint32_t n8 = len >> 3;
+    const float4* g4 = reinterpret_cast<const float4*>(g);
+    float4* x4 = reinterpret_cast<float4*>(x);
+    float4* m4 = reinterpret_cast<float4*>(m);
+    float4* v4 = reinterpret_cast<float4*>(v);
+    for (uint32_t i = tid; i < n8; i += NT) {
+        float4 G[2], X[2], M[2], V[2];
+#pragma unroll
+        for (int c2 = 0; c2 < 2; ++c2) {
+            G[c2] = ld_stream(g4 + 2 * i + c2); X[c2] = ld_stream(x4 + 2 * i + c2);
+            M[c2] = ld_stream(m4 + 2 * i + c2);
+            if (INNER == 0) V[c2] = ld_stream(v4 + 2 * i + c2);
+        }
+#pragma unroll
+        for (int c2 = 0; c2 < 2; ++c2) {
+            if (INNER == 0) { PALSGD_FOR4(adamw_elem(compv(G[c2], c), comp(X[c2], c), comp(M[c2], c), comp(V[c2], c), as)) }
+            else            { PALSGD_FOR4(sgdm_elem(compv(G[c2], c), comp(X[c2], c), comp(M[c2], c), ss)) }
+            st_stream(x4 + 2 * i + c2, X[c2]); st_stream(m4 + 2 * i + c2, M[c2]);
+            if (INNER == 0) st_stream(v4 + 2 * i + c2, V[c2]);
+        }
+    }
+    for (uint32_t i = (n8 << 3) + tid; i < len; i += NT) {
+        float xi = x[i], mi = m[i];
+        if (INNER == 0) { float vi = v[i]; adamw_elem(g[i], xi, mi, vi, as); v[i] = vi; }
+        else            { sgdm_elem(g[i], xi, mi, ss); }
+        x[i] = xi; m[i] = mi;
+    }
+}
+
+template <int NT>
+__device__ __forceinline__ void pull_chunk_f32_pair(uint32_t tid, float* __restrict__ x, const float* __restrict__ xg,
+                                                    uint32_t len, float beta)
+{
+    const uint32_t n8 = len >> 3;
+    float4* x4 = reinterpret_cast<float4*>(x);
+    const float4* q4 = reinterpret_cast<const float4*>(xg);
+    for (uint32_t i = tid; i < n8; i += NT) {
+        float4 X[2], Q[2];
+#pragma unroll
+        for (int c2 = 0; c2 < 2; ++c2) { X[c2] = ld_stream(x4 + 2 * i + c2); Q[c2] = __ldg(q4 + 2 * i + c2); }
+#pragma unroll
+        for (int c2 = 0; c2 < 2; ++c2) {
+            PALSGD_FOR4(comp(X[c2], c) = pull_elem(compv(X[c2], c), compv(Q[c2], c), beta))
+            st_stream(x4 + 2 * i + c2, X[c2]);
+        }
+    }
+    for (uint32_t i = (n8 << 3) + tid; i < len; i += NT) x[i] = pull_elem(x[i], xg[i], beta);
 }
 
 // ---------------------------------------------------------------- bf16 + fp32-master chunk bodies
@@ -172,8 +229,8 @@ __device__ __forceinline__ uint4 pack8(const float4& a, const float4& b)
                       pack_bf16x2(b.x, b.y), pack_bf16x2(b.z, b.w));
 }
 
-template <int U>
-__device__ __forceinline__ void adamw_chunk_bf16(const __nv_bfloat16* __restrict__ g,
+template <int U, int NT>
+__device__ __forceinline__ void adamw_chunk_bf16(uint32_t tid, const __nv_bfloat16* __restrict__ g,
                                                  __nv_bfloat16* __restrict__ w, float* __restrict__ x,
                                                  float* __restrict__ m, float* __restrict__ v,
                                                  uint32_t len, const AdamScalars& s)
@@ -184,11 +241,11 @@ __device__ __forceinline__ void adamw_chunk_bf16(const __nv_bfloat16* __restrict
     float4* x4 = reinterpret_cast<float4*>(x);
     float4* m4 = reinterpret_cast<float4*>(m);
     float4* v4 = reinterpret_cast<float4*>(v);
-    for (uint32_t base = 0; base < n8; base += kThreads * U) {
+    for (uint32_t base = 0; base < n8; base += NT * U) {
         uint4 G[U]; float4 X[U][2], M[U][2], V[U][2];
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-            const uint32_t i = base + u * kThreads + threadIdx.x;
+            const uint32_t i = base + u * NT + tid;
             if (i < n8) {
                 G[u] = ld_stream(g8 + i);
                 X[u][0] = ld_stream(x4 + 2 * i); X[u][1] = ld_stream(x4 + 2 * i + 1);
@@ -198,7 +255,7 @@ __device__ __forceinline__ void adamw_chunk_bf16(const __nv_bfloat16* __restrict
         }
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-            const uint32_t i = base + u * kThreads + threadIdx.x;
+            const uint32_t i = base + u * NT + tid;
             if (i < n8) {
                 float gf[8]; unpack8(G[u], gf);
                 PALSGD_FOR4(adamw_elem(gf[c],     comp(X[u][0], c), comp(M[u][0], c), comp(V[u][0], c), s))
@@ -210,14 +267,14 @@ __device__ __forceinline__ void adamw_chunk_bf16(const __nv_bfloat16* __restrict
             }
         }
     }
-    const uint32_t i = (n8 << 3) + threadIdx.x;
+    const uint32_t i = (n8 << 3) + tid;
     if (i < len) { float xi = x[i], mi = m[i], vi = v[i];
                    adamw_elem(__bfloat162float(g[i]), xi, mi, vi, s);
                    x[i] = xi; m[i] = mi; v[i] = vi; w[i] = __float2bfloat16_rn(xi); }
 }
 
-template <int U>
-__device__ __forceinline__ void sgdm_chunk_bf16(const __nv_bfloat16* __restrict__ g,
+template <int U, int NT>
+__device__ __forceinline__ void sgdm_chunk_bf16(uint32_t tid, const __nv_bfloat16* __restrict__ g,
                                                 __nv_bfloat16* __restrict__ w, float* __restrict__ x,
                                                 float* __restrict__ buf, uint32_t len, const SgdScalars& s)
 {
@@ -226,11 +283,11 @@ __device__ __forceinline__ void sgdm_chunk_bf16(const __nv_bfloat16* __restrict_
     uint4* w8 = reinterpret_cast<uint4*>(w);
     float4* x4 = reinterpret_cast<float4*>(x);
     float4* b4 = reinterpret_cast<float4*>(buf);
-    for (uint32_t base = 0; base < n8; base += kThreads * U) {
+    for (uint32_t base = 0; base < n8; base += NT * U) {
         uint4 G[U]; float4 X[U][2], B[U][2];
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-            const uint32_t i = base + u * kThreads + threadIdx.x;
+            const uint32_t i = base + u * NT + tid;
             if (i < n8) {
                 G[u] = ld_stream(g8 + i);
                 X[u][0] = ld_stream(x4 + 2 * i); X[u][1] = ld_stream(x4 + 2 * i + 1);
@@ -239,7 +296,7 @@ __device__ __forceinline__ void sgdm_chunk_bf16(const __nv_bfloat16* __restrict_
         }
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-            const uint32_t i = base + u * kThreads + threadIdx.x;
+            const uint32_t i = base + u * NT + tid;
             if (i < n8) {
                 float gf[8]; unpack8(G[u], gf);
                 PALSGD_FOR4(sgdm_elem(gf[c],     comp(X[u][0], c), comp(B[u][0], c), s))
@@ -250,30 +307,30 @@ __device__ __forceinline__ void sgdm_chunk_bf16(const __nv_bfloat16* __restrict_
             }
         }
     }
-    const uint32_t i = (n8 << 3) + threadIdx.x;
+    const uint32_t i = (n8 << 3) + tid;
     if (i < len) { float xi = x[i], bi = buf[i]; sgdm_elem(__bfloat162float(g[i]), xi, bi, s);
                    x[i] = xi; buf[i] = bi; w[i] = __float2bfloat16_rn(xi); }
 }
 
-template <int U>
-__device__ __forceinline__ void pull_chunk_bf16(__nv_bfloat16* __restrict__ w, float* __restrict__ x,
+template <int U, int NT>
+__device__ __forceinline__ void pull_chunk_bf16(uint32_t tid, __nv_bfloat16* __restrict__ w, float* __restrict__ x,
                                                 const float* __restrict__ xg, uint32_t len, float beta)
 {
     const uint32_t n8 = len >> 3;
     uint4* w8 = reinterpret_cast<uint4*>(w);
     float4* x4 = reinterpret_cast<float4*>(x);
     const float4* q4 = reinterpret_cast<const float4*>(xg);
-    for (uint32_t base = 0; base < n8; base += kThreads * U) {
+    for (uint32_t base = 0; base < n8; base += NT * U) {
         float4 X[U][2], Q[U][2];
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-            const uint32_t i = base + u * kThreads + threadIdx.x;
+            const uint32_t i = base + u * NT + tid;
             if (i < n8) { X[u][0] = ld_stream(x4 + 2 * i); X[u][1] = ld_stream(x4 + 2 * i + 1);
                           Q[u][0] = __ldg(q4 + 2 * i);      Q[u][1] = __ldg(q4 + 2 * i + 1); }
         }
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-            const uint32_t i = base + u * kThreads + threadIdx.x;
+            const uint32_t i = base + u * NT + tid;
             if (i < n8) {
                 PALSGD_FOR4(comp(X[u][0], c) = pull_elem(compv(X[u][0], c), compv(Q[u][0], c), beta))
                 PALSGD_FOR4(comp(X[u][1], c) = pull_elem(compv(X[u][1], c), compv(Q[u][1], c), beta))
@@ -282,17 +339,81 @@ __device__ __forceinline__ void pull_chunk_bf16(__nv_bfloat16* __restrict__ w, f
             }
         }
     }
-    const uint32_t i = (n8 << 3) + threadIdx.x;
+    const uint32_t i = (n8 << 3) + tid;
+    if (i < len) { const float xi = pull_elem(x[i], xg[i], beta); x[i] = xi; w[i] = __float2bfloat16_rn(xi); }
+}
+
+
+// ---- bf16 mode with 4-element units (64-bit accesses to the bf16 streams): fewer registers
+// per thread, so more CTAs are resident per SM.  Selected with U = 0 in grad_item / pull_item.
+__device__ __forceinline__ void unpack4(const uint2& h, float (&f)[4])
+{
+    f[0] = bf16_bits_to_f32(h.x & 0xFFFFu); f[1] = __uint_as_float(h.x & 0xFFFF0000u);
+    f[2] = bf16_bits_to_f32(h.y & 0xFFFFu); f[3] = __uint_as_float(h.y & 0xFFFF0000u);
+}
+__device__ __forceinline__ uint2 pack4(const float4& a)
+{
+    return make_uint2(pack_bf16x2(a.x, a.y), pack_bf16x2(a.z, a.w));
+}
+
+template <int INNER, int NT>
+__device__ __forceinline__ void grad_chunk_bf16_u4(uint32_t tid, const __nv_bfloat16* __restrict__ g,
+                                                   __nv_bfloat16* __restrict__ w, float* __restrict__ x,
+                                                   float* __restrict__ m, float* __restrict__ v, uint32_t len,
+                                                   const AdamScalars& as, const SgdScalars& ss)
+{
+    const uint32_t n4 = len >> 2;
+    const uint2* g4 = reinterpret_cast<const uint2*>(g);
+    uint2* w4 = reinterpret_cast<uint2*>(w);
+    float4* x4 = reinterpret_cast<float4*>(x);
+    float4* m4 = reinterpret_cast<float4*>(m);
+    float4* v4 = reinterpret_cast<float4*>(v);
+    for (uint32_t i = tid; i < n4; i += NT) {
+        const uint2 G = ld_stream(g4 + i);
+        float4 X = ld_stream(x4 + i), M = ld_stream(m4 + i), V;
+        if (INNER == 0) V = ld_stream(v4 + i);
+        float gf[4]; unpack4(G, gf);
+        if (INNER == 0) { PALSGD_FOR4(adamw_elem(gf[c], comp(X, c), comp(M, c), comp(V, c), as)) }
+        else            { PALSGD_FOR4(sgdm_elem(gf[c], comp(X, c), comp(M, c), ss)) }
+        st_stream(x4 + i, X); st_stream(m4 + i, M);
+        if (INNER == 0) st_stream(v4 + i, V);
+        st_stream(w4 + i, pack4(X));
+    }
+    const uint32_t i = (n4 << 2) + tid;
+    if (i < len) {
+        float xi = x[i], mi = m[i];
+        if (INNER == 0) { float vi = v[i]; adamw_elem(__bfloat162float(g[i]), xi, mi, vi, as); v[i] = vi; }
+        else            { sgdm_elem(__bfloat162float(g[i]), xi, mi, ss); }
+        x[i] = xi; m[i] = mi; w[i] = __float2bfloat16_rn(xi);
+    }
+}
+
+template <int NT>
+__device__ __forceinline__ void pull_chunk_bf16_u4(uint32_t tid, __nv_bfloat16* __restrict__ w, float* __restrict__ x,
+                                                   const float* __restrict__ xg, uint32_t len, float beta)
+{
+    const uint32_t n4 = len >> 2;
+    uint2* w4 = reinterpret_cast<uint2*>(w);
+    float4* x4 = reinterpret_cast<float4*>(x);
+    const float4* q4 = reinterpret_cast<const float4*>(xg);
+    for (uint32_t i = tid; i < n4; i += NT) {
+        float4 X = ld_stream(x4 + i);
+        const float4 Q = __ldg(q4 + i);
+        PALSGD_FOR4(comp(X, c) = pull_elem(compv(X, c), compv(Q, c), beta))
+        st_stream(x4 + i, X);
+        st_stream(w4 + i, pack4(X));
+    }
+    const uint32_t i = (n4 << 2) + tid;
     if (i < len) { const float xi = pull_elem(x[i], xg[i], beta); x[i] = xi; w[i] = __float2bfloat16_rn(xi); }
 }
 
 // ---------------------------------------------------------------- scalar bodies (unaligned segments)
 
-template <int INNER, int PREC>
-__device__ __forceinline__ void grad_chunk_scalar(const void* g, __nv_bfloat16* w, float* x, float* m, float* v,
+template <int INNER, int PREC, int NT>
+__device__ __forceinline__ void grad_chunk_scalar(uint32_t tid, const void* g, __nv_bfloat16* w, float* x, float* m, float* v,
                                                   uint32_t len, const AdamScalars& as, const SgdScalars& ss)
 {
-    for (uint32_t i = threadIdx.x; i < len; i += kThreads) {
+    for (uint32_t i = tid; i < len; i += NT) {
         const float gi = PREC ? __bfloat162float(static_cast<const __nv_bfloat16*>(g)[i])
                               : static_cast<const float*>(g)[i];
         float xi = x[i], mi = m[i];
@@ -303,10 +424,10 @@ __device__ __forceinline__ void grad_chunk_scalar(const void* g, __nv_bfloat16* 
     }
 }
 
-template <int PREC>
-__device__ __forceinline__ void pull_chunk_scalar(__nv_bfloat16* w, float* x, const float* xg, uint32_t len, float beta)
+template <int PREC, int NT>
+__device__ __forceinline__ void pull_chunk_scalar(uint32_t tid, __nv_bfloat16* w, float* x, const float* xg, uint32_t len, float beta)
 {
-    for (uint32_t i = threadIdx.x; i < len; i += kThreads) {
+    for (uint32_t i = tid; i < len; i += NT) {
         const float xi = pull_elem(x[i], xg[i], beta);
         x[i] = xi;
         if (PREC) w[i] = __float2bfloat16_rn(xi);
@@ -315,8 +436,8 @@ __device__ __forceinline__ void pull_chunk_scalar(__nv_bfloat16* w, float* x, co
 
 // ---------------------------------------------------------------- dispatch of one work item
 
-template <int PREC, int U>
-__device__ __forceinline__ void pull_item(const Tables& tb, uint32_t k, const Chunk& ch, float beta)
+template <int PREC, int U, int NT>
+__device__ __forceinline__ void pull_item(uint32_t tid, const Tables& tb, uint32_t k, const Chunk& ch, float beta)
 {
     const uint32_t seg = ch.seg & ~kSegVecFlag;
     const size_t   pi  = (size_t)k * tb.n_seg + seg;
@@ -324,15 +445,17 @@ __device__ __forceinline__ void pull_item(const Tables& tb, uint32_t k, const Ch
     const float* xg = tb.global[seg] + ch.off;
     __nv_bfloat16* w = PREC ? tb.xw[pi] + ch.off : nullptr;
     if (ch.seg & kSegVecFlag) {
-        if (PREC) pull_chunk_bf16<U>(w, x, xg, ch.len, beta);
-        else      pull_chunk_f32<U>(x, xg, ch.len, beta);
+        if (PREC && U == 0) pull_chunk_bf16_u4<NT>(tid, w, x, xg, ch.len, beta);
+        else if (PREC) pull_chunk_bf16<(U > 0 ? U : 1), NT>(tid, w, x, xg, ch.len, beta);
+        else if (U == -1) pull_chunk_f32_pair<NT>(tid, x, xg, ch.len, beta);
+        else      pull_chunk_f32<(U > 0 ? U : 1), NT>(tid, x, xg, ch.len, beta);
     } else {
-        pull_chunk_scalar<PREC>(w, x, xg, ch.len, beta);
+        pull_chunk_scalar<PREC, NT>(tid, w, x, xg, ch.len, beta);
     }
 }
 
-template <int INNER, int PREC, int U>
-__device__ __forceinline__ void grad_item(const Tables& tb, uint32_t k, const Chunk& ch,
+template <int INNER, int PREC, int U, int NT>
+__device__ __forceinline__ void grad_item(uint32_t tid, const Tables& tb, uint32_t k, const Chunk& ch,
                                           const AdamScalars& as, const SgdScalars& ss)
 {
     const uint32_t seg = ch.seg & ~kSegVecFlag;
@@ -344,18 +467,20 @@ __device__ __forceinline__ void grad_item(const Tables& tb, uint32_t k, const Ch
         const __nv_bfloat16* g = static_cast<const __nv_bfloat16*>(tb.grad[pi]) + ch.off;
         __nv_bfloat16* w = tb.xw[pi] + ch.off;
         if (ch.seg & kSegVecFlag) {
-            if (INNER == 0) adamw_chunk_bf16<U>(g, w, x, m, v, ch.len, as);
-            else            sgdm_chunk_bf16<U>(g, w, x, m, ch.len, ss);
+            if (U == 0)          grad_chunk_bf16_u4<INNER, NT>(tid, g, w, x, m, v, ch.len, as, ss);
+            else if (INNER == 0) adamw_chunk_bf16<(U > 0 ? U : 1), NT>(tid, g, w, x, m, v, ch.len, as);
+            else                 sgdm_chunk_bf16<(U > 0 ? U : 1), NT>(tid, g, w, x, m, ch.len, ss);
         } else {
-            grad_chunk_scalar<INNER, 1>(g, w, x, m, v, ch.len, as, ss);
+            grad_chunk_scalar<INNER, 1, NT>(tid, g, w, x, m, v, ch.len, as, ss);
         }
     } else {
         const float* g = static_cast<const float*>(tb.grad[pi]) + ch.off;
         if (ch.seg & kSegVecFlag) {
-            if (INNER == 0) adamw_chunk_f32<U>(g, x, m, v, ch.len, as);
-            else            sgdm_chunk_f32<U>(g, x, m, ch.len, ss);
+            if (U == -1)         grad_chunk_f32_pair<INNER, NT>(tid, g, x, m, v, ch.len, as, ss);
+            else if (INNER == 0) adamw_chunk_f32<(U > 0 ? U : 1), NT>(tid, g, x, m, v, ch.len, as);
+            else                 sgdm_chunk_f32<(U > 0 ? U : 1), NT>(tid, g, x, m, ch.len, ss);
         } else {
-            grad_chunk_scalar<INNER, 0>(g, nullptr, x, m, v, ch.len, as, ss);
+            grad_chunk_scalar<INNER, 0, NT>(tid, g, nullptr, x, m, v, ch.len, as, ss);
         }
     }
 }
@@ -391,14 +516,14 @@ palsgd_inner_kernel(const __grid_constant__ InnerArgs a)
 
     const uint64_t n_items = (uint64_t)tb.n_chunks * K;
     for (uint64_t item = blockIdx.x; item < n_items; item += gridDim.x) {
-        const uint32_t k = (uint32_t)(item % K);
-        const Chunk ch = tb.chunks[item / K];
+        const uint32_t k = (uint32_t)(a.chunk_major ? item / tb.n_chunks : item % K);
+        const Chunk ch = tb.chunks[a.chunk_major ? item % tb.n_chunks : item / K];
         if (s_pull[k]) {
-            pull_item<PREC, U>(tb, k, ch, a.beta_pull);
+            pull_item<PREC, U, kThreads>(threadIdx.x, tb, k, ch, a.beta_pull);
         } else {
             const AdamScalars as{a.b1, a.b2, a.omb1, a.omb2, s_bc1[k], s_bc2[k], a.decay, a.lr, a.eps};
             const SgdScalars  ss{a.mu, a.wd, a.lr};
-            grad_item<INNER, PREC, U>(tb, k, ch, as, ss);
+            grad_item<INNER, PREC, U, kThreads>(threadIdx.x, tb, k, ch, as, ss);
         }
     }
 
@@ -433,7 +558,7 @@ palsgd_pull_kernel(const __grid_constant__ PullArgs a)
     const uint64_t n_items = (uint64_t)tb.n_chunks * K;
     for (uint64_t item = blockIdx.x; item < n_items; item += gridDim.x) {
         const uint32_t k = (uint32_t)(item % K);
-        if ((a.mask >> k) & 1ull) pull_item<PREC, U>(tb, k, tb.chunks[item / K], a.beta);
+        if ((a.mask >> k) & 1ull) pull_item<PREC, U, kThreads>(threadIdx.x, tb, k, tb.chunks[item / K], a.beta);
     }
 }
 
@@ -461,8 +586,13 @@ palsgd_outer_kernel(const __grid_constant__ OuterArgs a)
     const uint32_t K = tb.K;
     constexpr int B = 8;                                   // slot loads issued together
 
-    for (uint32_t c = blockIdx.x; c < tb.n_chunks; c += gridDim.x) {
-        const Chunk ch = tb.chunks[c];
+    const uint64_t n_items = (uint64_t)tb.n_chunks * a.parts;
+    for (uint64_t item = blockIdx.x; item < n_items; item += gridDim.x) {
+        Chunk ch = tb.chunks[item / a.parts];
+        const uint32_t begin = (uint32_t)(item % a.parts) * a.sub_elems;      // this item's slice of the chunk
+        if (begin >= ch.len) continue;                                        // uniform over the CTA
+        ch.off += begin;
+        ch.len = min(ch.len - begin, a.sub_elems);
         const uint32_t seg = ch.seg & ~kSegVecFlag;
         __syncthreads();
         if (threadIdx.x < K) {

@@ -178,6 +178,28 @@ def test_run_to_run_determinism_and_launch_shape_independence():
             assert np.array_equal(outs[0][k], o[k]), k
 
 
+@pytest.mark.parametrize("variant,stages,cap", [(10, 0, 0), (11, 0, 0), (12, 0, 0), (10, 2, 3), (11, 3, 1), (12, 2, 2),
+                                                (3, 0, 0), (5, 0, 5), (7, 0, 0), (9, 0, 0), (13, 0, 0), (15, 0, 9)])
+@pytest.mark.parametrize("inner,precision", [(0, 0), (1, 0), (0, 1), (1, 1)])
+def test_every_compiled_form_of_the_inner_kernel_matches_oracle(variant, stages, cap, inner, precision):
+    # 10/11: persistent shared-memory-ring form (full chunks through the ring, the rest by registers)
+    numel = [4096 * 37 + 11, 5, 4096 * 2, 1001]
+    P = sum(numel)
+    cfg = _cfg(numel, K=5, H=3, T=7, p=0.3, inner=inner, precision=precision,
+               momentum=0.9 if inner else 0.0)
+    x0 = _x0(cfg.K, P, seed=5)
+    for layout in ("arena", "separate"):
+        gpu, orc = GpuRun(cfg, x0, numel=numel, layout=layout), make_oracle(cfg, x0)
+        gpu.lib.set_tuning(2, variant); gpu.lib.set_tuning(3, stages); gpu.lib.set_tuning(0, cap)
+        for t in range(cfg.T):
+            g = _grads(cfg, P, t)
+            gpu.set_grads(g); gpu.step(cfg.lr, cfg.eta); orc.step(g, cfg.lr, cfg.eta)
+        compare_state(gpu.state(), orc, exact=True)
+        c = gpu.counters()                       # also raises if a bounded wait expired
+        assert c["s"] == [int(v) for v in orc.s] and c["t"] == cfg.T
+        assert gpu.guards_intact()
+
+
 def test_step_host_moves_gradients_and_results_through_host_buffers():
     numel = [5000, 37, 4096]
     P = sum(numel)
