@@ -50,6 +50,31 @@ def measured_peak_gbs():
         return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
 
 
+# DRAM traffic (ncu: dram__bytes_read.sum + dram__bytes_write.sum) divided by the algorithmic bytes
+# of the same launch, measured on the 16M-element stand-ins of the same kernels (all-gradient inner
+# launch; outer launch).  Traffic grows in proportion to the elements processed, so the ratio carries
+# over to the full-size launch.  Valid only for the kernel sources with the digest recorded here.
+NCU_TRAFFIC = {"digest": "89d23b06744ff9e3",
+               "inner": {0: 0.985, 1: 0.985},      # by precision: fp32, bf16 + fp32 master
+               "outer": {0: 0.957, 1: 0.964}}
+
+
+def kernel_digest() -> str:
+    import hashlib
+    h = hashlib.sha256()
+    for f in ("palsgd_device.cuh", "palsgd_kernels.cuh"):
+        with open(os.path.join(ROOT, "paper_2504_18454_b200", "csrc", f), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
+
+
+def ncu_traffic(kind: str, precision: int, alg_bytes_per_launch):
+    """Measured DRAM bytes per launch, or None once the kernels changed since the capture."""
+    if alg_bytes_per_launch is None or kernel_digest() != NCU_TRAFFIC["digest"]:
+        return None
+    return NCU_TRAFFIC[kind][precision] * alg_bytes_per_launch
+
+
 def inner_bytes_per_element(cfg, pull: bool) -> int:
     """Algorithmic HBM bytes per worker-element of the fused inner kernel."""
     bf = cfg.precision == 1
@@ -331,13 +356,15 @@ def run_ours(args, cfg):
             "data": "synthetic", "config": workload_config(cfg, args),
             "roofline": {"bound": "hbm", "kernel": "palsgd_inner_kernel", "achieved": inner_gbs,
                          "peak": peak, "unit": "GB/s", "frac": inner_gbs / peak if inner_gbs else None,
-                         "traffic": None, "peak_source": peak_src, "frac_of_8000_nominal":
+                         "traffic": ncu_traffic("inner", cfg.precision, inner_bytes / n_inner if n_inner else None),
+                         "peak_source": peak_src, "frac_of_8000_nominal":
                          inner_gbs / 8000.0 if inner_gbs else None,
                          "launches": n_inner, "avg_ms": inner_ms / n_inner if n_inner else None,
                          "alg_bytes_per_launch": inner_bytes / n_inner if n_inner else None},
             "roofline_outer": {"bound": "hbm", "kernel": "palsgd_outer_kernel", "achieved": outer_gbs,
                                "peak": peak, "unit": "GB/s", "frac": outer_gbs / peak if outer_gbs else None,
-                               "traffic": None, "frac_of_8000_nominal": outer_gbs / 8000.0 if outer_gbs else None,
+                               "traffic": ncu_traffic("outer", cfg.precision, outer_bytes / n_outer if n_outer else None),
+                               "frac_of_8000_nominal": outer_gbs / 8000.0 if outer_gbs else None,
                                "launches": n_outer, "avg_ms": outer_ms / n_outer if n_outer else None,
                                "alg_bytes_per_launch": outer_bytes / n_outer if n_outer else None,
                                "params_per_s": Pn * n_outer / (outer_ms * 1e-3) if outer_ms else None},

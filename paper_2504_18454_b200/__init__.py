@@ -19,4 +19,6 @@ from .binding import (  # noqa: F401
     TUNE_OUTER_GRID_CAP,
     TUNE_INNER_VARIANT,
     TUNE_PIPE_STAGES,
+    TUNE_CHUNK_MAJOR,
+    TUNE_OUTER_SUB_ELEMS,
 )

@@ -11,6 +11,7 @@ LIB_PATH = HERE / "libpalsgd.so"
 INNER_ADAMW, INNER_SGDM = 0, 1
 PREC_FP32, PREC_BF16_MASTER = 0, 1
 TUNE_INNER_GRID_CAP, TUNE_OUTER_GRID_CAP, TUNE_INNER_VARIANT, TUNE_PIPE_STAGES = 0, 1, 2, 3
+TUNE_CHUNK_MAJOR, TUNE_OUTER_SUB_ELEMS = 4, 5
 MAX_WORKERS = 64
 
 
