@@ -56,7 +56,8 @@ typedef enum palsgd_status {
     PALSGD_ESTATE       = -4,   /* call not valid in this state (e.g. undefined coefficient)         */
     PALSGD_ENOMEM       = -5,   /* host or device allocation failed                                  */
     PALSGD_EUNSUPPORTED = -6,   /* combination not built                                             */
-    PALSGD_ETIMEOUT     = -7    /* a bounded wait inside a kernel expired (reported by get_counters)  */
+    PALSGD_ETIMEOUT     = -7,   /* a bounded wait inside a kernel expired (reported by get_counters)  */
+    PALSGD_ETOOBIG      = -8    /* tensor list needs more than the fixed scratch of a no-allocation call */
 } palsgd_status;
 
 enum { PALSGD_INNER_ADAMW = 0, PALSGD_INNER_SGDM = 1 };
@@ -208,6 +209,55 @@ int palsgd_decision(uint64_t seed, uint64_t t, uint32_t k, double p);
 /* Text for a status; the CUDA error string of the latest ECUDA on ctx (or ""). */
 const char* palsgd_strerror(int status);
 const char* palsgd_last_cuda_error(palsgd_ctx* ctx);
+
+/*
+ * Outer synchronisation WITHOUT any allocation (the paper has no counterpart:
+ * this entry point exists for the way the library gets embedded, not for the
+ * method).  Same arithmetic, same kernel and same results as palsgd_outer_sync,
+ * for callers that are not allowed to allocate device memory at the point where
+ * they synchronise: code running inside a framework whose caching allocator
+ * owns all of the GPU's memory, inside a region where cudaMalloc's implicit
+ * device-wide synchronisation is unacceptable, or in a process whose memory
+ * budget is fixed up front.  Such callers cannot use palsgd_init, which
+ * allocates the launch tables.  Here the tables live in a fixed array of
+ * PALSGD_NOALLOC_SCRATCH_BYTES that is part of the library image: every GPU
+ * that loads the library holds that much memory until the process exits.
+ *
+ * No context: the caller passes the buffers on every call.  Layout as in
+ * palsgd_buffers: param/master are [K*n_tensors] device pointers indexed
+ * [k*n_tensors + j], global/outer_mom are [n_tensors]; the pointer ARRAYS are
+ * host memory.  FP32: param = float local models, master = NULL.  BF16_MASTER:
+ * master = fp32 local models (averaged and rewritten), param = bf16 working
+ * copies (rewritten as RNE of the new global model).  numel[j] = 0 is allowed.
+ * The call rebuilds the tables, copies them into the array on `stream`, and
+ * launches one kernel on `stream`; it does not synchronise.  It calls neither
+ * cudaMalloc nor cudaFree nor any other allocating routine, on the device or on
+ * the host.
+ *
+ * Limit: the tables need 16 bytes per started block of 8192 elements of every
+ * tensor, plus 8 bytes per (worker, non-empty tensor) pointer (twice that in
+ * BF16_MASTER mode) and 16 bytes per non-empty tensor, each table rounded up to
+ * 256 bytes.  If that exceeds PALSGD_NOALLOC_SCRATCH_BYTES the call returns
+ * PALSGD_ETOOBIG and does nothing (1 MiB covers about 5*10^8 parameters in a
+ * few hundred tensors at K = 8).
+ *
+ * Sharing: all calls on a device use the one array, and it keeps the previous
+ * call's tables.  Each call overwrites everything it will read, so nothing has
+ * to be cleared; but two calls whose GPU work can overlap (different streams
+ * without an ordering between them, or several host threads on different
+ * streams) race on the array and give undefined results.  Order them on one
+ * stream, or with events.  Host threads are serialised inside the call.
+ *
+ * First call on each device: looks up the array's device address (a runtime
+ * call that is made once per device and cached, with that device current).
+ * Make this first call outside any stream capture.
+ * Errors: EINVAL, EALIGN, ETOOBIG before any CUDA call; ECUDA.
+ */
+#define PALSGD_NOALLOC_SCRATCH_BYTES (1u << 20)
+int palsgd_outer_sync_noalloc(uint32_t K, int32_t precision, size_t n_tensors,
+                              const uint64_t* numel, void* const* param, float* const* master,
+                              float* const* global, float* const* outer_mom, double outer_lr,
+                              double outer_momentum, int32_t outer_nesterov, void* stream);
 
 /* Free the context and its device tables.  NULL is accepted.  The caller's
  * buffers are not touched. */

@@ -9,6 +9,8 @@ from .binding import (  # noqa: F401
     Palsgd,
     PalsgdError,
     decision,
+    outer_sync_noalloc,
+    NOALLOC_SCRATCH_BYTES,
     lib,
     strerror,
     INNER_ADAMW,

@@ -66,6 +66,9 @@ def lib() -> C.CDLL:
                  "palsgd_step", "palsgd_step_host", "palsgd_get_counters", "palsgd_set_counters",
                  "palsgd_get_launch_count", "palsgd_set_tuning", "palsgd_decision"):
         getattr(L, name).restype = C.c_int
+    L.palsgd_outer_sync_noalloc.argtypes = [C.c_uint32, C.c_int32, C.c_size_t, u64p, C.POINTER(vp), C.POINTER(vp),
+                                            C.POINTER(vp), C.POINTER(vp), C.c_double, C.c_double, C.c_int32, vp]
+    L.palsgd_outer_sync_noalloc.restype = C.c_int
     L.palsgd_strerror.argtypes = [C.c_int]
     L.palsgd_strerror.restype = C.c_char_p
     L.palsgd_last_cuda_error.argtypes = [vp]
@@ -95,6 +98,29 @@ def _ptr_array(ptrs: Sequence[int]):
 def _data_ptrs(per_worker: Sequence[Sequence]) -> List[int]:
     """[k][j] tensors (anything with .data_ptr()) -> flat [k*n + j] addresses."""
     return [int(t.data_ptr()) for row in per_worker for t in row]
+
+
+NOALLOC_SCRATCH_BYTES = 1 << 20
+
+
+def outer_sync_noalloc(*, K: int, numel: Sequence[int], params, global_, outer_mom, master=None,
+                       outer_lr: float = 0.7, outer_momentum: float = 0.9, outer_nesterov: bool = True,
+                       precision: int = PREC_FP32, stream: int = 0) -> None:
+    """palsgd_outer_sync_noalloc: the outer synchronisation for callers that may not allocate
+    device memory (no context; the launch tables go into a fixed array inside the library).
+    params/master: K lists of n tensors; global_/outer_mom: n tensors.  Calls whose GPU work
+    could overlap race on that array: keep them on one stream."""
+    n = len(numel)
+    nm = (C.c_uint64 * n)(*[int(x) for x in numel])
+    cast = lambda a: C.cast(a, C.POINTER(C.c_void_p))
+    rc = lib().palsgd_outer_sync_noalloc(
+        int(K), int(precision), n, nm, cast(_ptr_array(_data_ptrs(params))),
+        cast(_ptr_array(_data_ptrs(master))) if master is not None else None,
+        cast(_ptr_array([int(t.data_ptr()) for t in global_])),
+        cast(_ptr_array([int(t.data_ptr()) for t in outer_mom])),
+        float(outer_lr), float(outer_momentum), int(bool(outer_nesterov)), C.c_void_p(stream))
+    if rc:
+        raise PalsgdError(rc, "palsgd_outer_sync_noalloc")
 
 
 class Palsgd:

@@ -14,7 +14,7 @@ from pathlib import Path
 HERE = Path(__file__).resolve().parent
 CSRC = HERE / "csrc"
 LIB = HERE / "libpalsgd.so"
-SOURCES = [CSRC / "palsgd_api.cu"]
+SOURCES = [CSRC / "palsgd_api.cu", CSRC / "palsgd_noalloc.cu"]
 DEPS = sorted(CSRC.glob("*.cu*")) + [HERE.parent / "include" / "palsgd.h", Path(__file__)]
 
 NVCC_FLAGS = [

@@ -642,6 +642,7 @@ extern "C" const char* palsgd_strerror(int status)
         case PALSGD_ENOMEM: return "out of memory";
         case PALSGD_EUNSUPPORTED: return "unsupported combination";
         case PALSGD_ETIMEOUT: return "a bounded device-side wait expired";
+        case PALSGD_ETOOBIG: return "tensor list exceeds the fixed scratch of the no-allocation entry point";
         default: return "unknown status";
     }
 }
