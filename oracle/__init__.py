@@ -163,12 +163,14 @@ class Oracle:
         self._pull = getattr(L, f"palsgd_oracle_pseudo_sync_{sfx}")
         self._outer = getattr(L, f"palsgd_oracle_outer_sync_{sfx}")
         self._step = getattr(L, f"palsgd_oracle_step_{sfx}")
+        self._ddp = getattr(L, f"palsgd_oracle_ddp_step_{sfx}")
         SP = C.POINTER(S)
         self._init.argtypes = [SP]; self._init.restype = None
         for f in (self._inner, self._step):
             f.argtypes = [SP, C.c_void_p, C.c_double, C.c_double, C.c_void_p]
             f.restype = C.c_int
         self._pull.argtypes = [SP, C.c_uint64, C.c_double]; self._pull.restype = None
+        self._ddp.argtypes = [SP, C.c_void_p, C.c_double]; self._ddp.restype = None
         self._outer.argtypes = [SP]; self._outer.restype = None
         self.precision = precision
         self._init(C.byref(self._st))
@@ -209,6 +211,11 @@ class Oracle:
         rc = self._step(C.byref(self._st), gp, float(lr_t), float(eta_t), fp)
         if rc:
             raise ValueError("undefined coefficient: pull with p=0 or gradient step with p=1")
+
+    def ddp_step(self, grads, lr_t: float) -> None:
+        """One step of the DDP warm-up phase: averaged gradient, one InnerOPT step for all workers."""
+        g, gp = self._grads_ptr(grads)
+        self._ddp(C.byref(self._st), gp, float(lr_t))
 
     def pseudo_sync(self, worker_mask: int, beta: float) -> None:
         self._pull(C.byref(self._st), int(worker_mask), float(beta))

@@ -16,6 +16,7 @@
  *   Algorithm 1 / Eq. (1), gradient step-> adamw_worker / sgdm_worker with
  *                                          step size alpha_t / (1 - p)
  *   Sec. 2.2 average, Eq. (3), Eq. (4)  -> FN(outer_sync)
+ *   Sec. 3.3 / Sec. 4.1 DDP warm-up     -> FN(ddp_step)
  *
  * The paper names its optimizers without printing them (Sec. 4.3): InnerOPT is
  * AdamW (decoupled weight decay, bias-corrected) or momentum SGD, OuterOPT is
@@ -243,6 +244,72 @@ void FN(outer_sync)(FN(state) *st)
     }
     for (uint32_t k = 0; k < K; ++k) refresh_working(st, k);
     st->n_outer += 1;
+}
+
+/* DDP warm-up step (Sec. 3.3 "we initialize training with a DDP warm-up phase";
+ * Sec. 4.1: Local SGD, DiLoCo and PALSGD all use DDP during the initial steps).
+ * Mini-batch SGD over K workers: the gradients are averaged,
+ *     gbar = (g_0 + g_1 + ... + g_{K-1}) / K      (ascending k, one division),
+ * and every worker applies the same InnerOPT step with the plain step size
+ * alpha_t (no 1/(1-p) rescaling: there is no mixing branch in this phase).
+ * In this phase all workers hold the same model and the same optimizer state;
+ * the step is therefore taken once, on worker 0's model and state, and the
+ * result is written to every worker, and to the global model copy x, which in
+ * this phase is that common model.  s_k and the bias-correction products of
+ * every worker follow worker 0.  No draw is made; the decisions of the step are
+ * recorded as 0; t advances; no outer synchronisation happens in this phase.
+ * grads: [K][P], float32 (mode 0) or bf16 bits (mode 1). */
+void FN(ddp_step)(FN(state) *st, const void *grads, double alpha_t)
+{
+    const uint32_t K = st->K;
+    const size_t P = st->P;
+    const float *g32 = st->precision == 0 ? (const float *)grads : NULL;
+    const uint16_t *g16 = st->precision == 1 ? (const uint16_t *)grads : NULL;
+    REAL *x = st->x, *m = st->m, *v = st->v;          /* worker 0 */
+
+    st->s[0] += 1;
+    if (st->inner == 0) { st->pow1[0] *= st->beta1; st->pow2[0] *= st->beta2; }
+    const REAL lr    = (REAL)alpha_t;
+    const REAL b1    = (REAL)st->beta1,         b2    = (REAL)st->beta2;
+    const REAL omb1  = (REAL)(1.0 - st->beta1), omb2  = (REAL)(1.0 - st->beta2);
+    const REAL bc1   = (REAL)(1.0 - st->pow1[0]);
+    const REAL bc2   = (REAL)(1.0 - st->pow2[0]);
+    const REAL decay = (REAL)(1.0 - alpha_t * st->weight_decay);
+    const REAL eps   = (REAL)st->eps;
+    const REAL mu    = (REAL)st->momentum, wd = (REAL)st->weight_decay;
+
+    #pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < (int64_t)P; ++i) {
+        REAL sum = g32 ? (REAL)g32[i] : (REAL)palsgd_oracle_bf16_to_f32(g16[i]);
+        for (uint32_t k = 1; k < K; ++k)
+            sum = sum + (g32 ? (REAL)g32[(size_t)k * P + i]
+                             : (REAL)palsgd_oracle_bf16_to_f32(g16[(size_t)k * P + i]));
+        REAL g = sum / (REAL)K;
+        REAL xi;
+        if (st->inner == 0) {
+            REAL mi = b1 * m[i] + omb1 * g;
+            REAL vi = b2 * v[i] + omb2 * (g * g);
+            REAL mhat = mi / bc1;
+            REAL vhat = vi / bc2;
+            xi = x[i] * decay;
+            REAL root = sizeof(REAL) == 4 ? (REAL)sqrtf((float)vhat) : (REAL)sqrt((double)vhat);
+            xi = xi - lr * (mhat / (root + eps));
+            for (uint32_t k = 0; k < K; ++k) { m[(size_t)k * P + i] = mi; v[(size_t)k * P + i] = vi; }
+        } else {
+            REAL gp = g + wd * x[i];
+            REAL b = mu * m[i] + gp;
+            xi = x[i] - lr * b;
+            for (uint32_t k = 0; k < K; ++k) m[(size_t)k * P + i] = b;
+        }
+        for (uint32_t k = 0; k < K; ++k) x[(size_t)k * P + i] = xi;
+        st->xg[i] = xi;
+    }
+    for (uint32_t k = 0; k < K; ++k) {
+        st->s[k] = st->s[0]; st->pow1[k] = st->pow1[0]; st->pow2[k] = st->pow2[0];
+        st->last_b[k] = 0;
+        refresh_working(st, k);
+    }
+    st->t += 1;
 }
 
 /* Algorithm 1, one iteration t: inner loop body, then "if (t+1) mod H = 0". */
