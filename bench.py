@@ -85,6 +85,12 @@ def inner_bytes_per_element(cfg, pull: bool) -> int:
     return 18 if bf else 20        # momentum SGD: read g, x, buf; write x, buf
 
 
+def ddp_bytes_per_param(cfg) -> int:
+    """DDP warm-up step: read K gradients and worker 0's x, m(, v); write x, m(, v) of all K slots
+    (+ K bf16 working copies) and x_g.  16K+16 (AdamW) or 12K+12 (momentum SGD) in both precisions."""
+    return (16 if cfg.inner == 0 else 12) * (cfg.K + 1)
+
+
 def outer_bytes_per_param(cfg) -> int:
     """Read K slots, x_g, u; write x_g, u, K slots (+ K bf16 working copies)."""
     return (10 if cfg.precision == 1 else 8) * cfg.K + 16
@@ -336,6 +342,20 @@ def run_ours(args, cfg):
         e2e = {"ms": ms_e2e, "steps": e2e_steps, "syncs": syncs,
                "h2d": K * Pn * es, "d2h": K + syncs * Pn * 4 / e2e_steps}
 
+    # ---- DDP warm-up kernel (the phase before Algorithm 1), timed on its own after the main regions
+    ddp = None
+    if not args.no_ddp:
+        for _ in range(3):
+            ctx.ddp_step(cfg.lr, stream)
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(9)]
+        evs[0].record()
+        for i in range(8):
+            ctx.ddp_step(cfg.lr, stream)
+            evs[i + 1].record()
+        torch.cuda.synchronize(dev)
+        ddp_ms = sum(evs[i].elapsed_time(evs[i + 1]) for i in range(8)) / 8
+        ddp = {"avg_ms": ddp_ms, "alg_bytes_per_launch": ddp_bytes_per_param(cfg) * Pn, "launches": 8}
+
     # ---- max over ranks
     if world > 1:
         t = torch.tensor([ms_total, e2e["ms"] if e2e else 0.0], device=dev, dtype=torch.float64)
@@ -368,6 +388,14 @@ def run_ours(args, cfg):
                                "launches": n_outer, "avg_ms": outer_ms / n_outer if n_outer else None,
                                "alg_bytes_per_launch": outer_bytes / n_outer if n_outer else None,
                                "params_per_s": Pn * n_outer / (outer_ms * 1e-3) if outer_ms else None},
+            "roofline_ddp": ({"bound": "hbm", "kernel": "palsgd_ddp_kernel",
+                              "achieved": ddp["alg_bytes_per_launch"] / (ddp["avg_ms"] * 1e-3) / 1e9,
+                              "peak": peak, "unit": "GB/s",
+                              "frac": ddp["alg_bytes_per_launch"] / (ddp["avg_ms"] * 1e-3) / 1e9 / peak,
+                              "traffic": None, "launches": ddp["launches"], "avg_ms": ddp["avg_ms"],
+                              "alg_bytes_per_launch": ddp["alg_bytes_per_launch"],
+                              "params_per_s": Pn / (ddp["avg_ms"] * 1e-3),
+                              "note": "timed outside the step loop; not part of value"} if ddp else None),
             "cpu_baseline": cpu_baseline,
             "e2e": ({"value": world * K * Pn * e2e["steps"] / (e2e["ms"] * 1e-3), "unit": UNIT,
                      "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
@@ -392,6 +420,7 @@ def main():
     ap.add_argument("--inner-variant", type=int, default=0, help="palsgd_set_tuning(INNER_VARIANT); 0 = default")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-ddp", action="store_true", help="skip the separate timing of the DDP warm-up kernel")
     args = ap.parse_args()
     cfg = W.get_config(args.workload)
     if args.impl == "reference":

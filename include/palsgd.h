@@ -128,6 +128,25 @@ int palsgd_init(palsgd_ctx** out, const palsgd_config* cfg, size_t n_tensors,
 int palsgd_inner_step(palsgd_ctx* ctx, double lr_t, double eta_t, void* stream);
 
 /*
+ * One step of the DDP warm-up phase that precedes Algorithm 1 (Sec. 3.3: training
+ * starts with a DDP phase; Sec. 4.1: all Local SGD variants use DDP for the initial
+ * steps), ONE kernel launch.  Mini-batch SGD over the K workers:
+ *   gbar = (g_0 + g_1 + ... + g_{K-1}) / K          (that order, one division)
+ *   one InnerOPT step with the plain step size lr = fl32(alpha_t) -- no 1/(1-p)
+ *   rescaling, there is no mixing branch in this phase -- using the formulas of
+ *   palsgd_inner_step's b = 0 case with g = gbar.
+ * In this phase all workers hold the same model and optimizer state, so the step
+ * is taken once, on worker 0's x, m, v and step count, and the result is written
+ * to every worker's x, m, v (and bf16 working copy) and to the global model copy
+ * x_g; s_k and the bias-correction products of every worker follow worker 0.
+ * The outer momentum u is not touched.  No draw; the recorded decisions are 0;
+ * t += 1 (the decision stream stays indexed by the global step).  Never runs the
+ * outer sync: switch to palsgd_step when the warm-up ends.
+ * Errors: EINVAL (NULL ctx, non-finite or negative rate); ECUDA.
+ */
+int palsgd_ddp_step(palsgd_ctx* ctx, double lr_t, void* stream);
+
+/*
  * A pull imposed on the workers whose bit is set in worker_mask, with the mixing
  * coefficient given directly (the EMA form after Eq. (2): x_k <- (1-beta) x_k +
  * beta x, computed as x - beta*(x - x_g)).  No draw; t, s_k unchanged.
@@ -195,11 +214,13 @@ int palsgd_get_launch_count(palsgd_ctx* ctx, uint64_t* n_launches);
  * kernel: 0 = worker index fastest (default), 1 = chunk index fastest.
  * OUTER_SUB_ELEMS: elements per work item of the outer kernel (a slice of a chunk),
  * a multiple of 1024; default 1024.
+ * DDP_SUB_ELEMS: the same for the DDP warm-up kernel; default 2048.
  * (Environment variable PALSGD_CHUNK_ELEMS, read by palsgd_init: elements per chunk
  * = per work item of the inner kernel, a multiple of 1024; default 4096 for fp32 AdamW,
  * 8192 otherwise.) */
 enum { PALSGD_TUNE_INNER_GRID_CAP = 0, PALSGD_TUNE_OUTER_GRID_CAP = 1, PALSGD_TUNE_INNER_VARIANT = 2,
-       PALSGD_TUNE_PIPE_STAGES = 3, PALSGD_TUNE_CHUNK_MAJOR = 4, PALSGD_TUNE_OUTER_SUB_ELEMS = 5 };
+       PALSGD_TUNE_PIPE_STAGES = 3, PALSGD_TUNE_CHUNK_MAJOR = 4, PALSGD_TUNE_OUTER_SUB_ELEMS = 5,
+       PALSGD_TUNE_DDP_SUB_ELEMS = 6 };
 int palsgd_set_tuning(palsgd_ctx* ctx, int knob, int64_t value);
 
 /* The branch draw as a pure host function: 1 = pseudo-sync, 0 = gradient step;

@@ -23,4 +23,5 @@ from .binding import (  # noqa: F401
     TUNE_PIPE_STAGES,
     TUNE_CHUNK_MAJOR,
     TUNE_OUTER_SUB_ELEMS,
+    TUNE_DDP_SUB_ELEMS,
 )

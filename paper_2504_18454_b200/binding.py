@@ -11,7 +11,7 @@ LIB_PATH = HERE / "libpalsgd.so"
 INNER_ADAMW, INNER_SGDM = 0, 1
 PREC_FP32, PREC_BF16_MASTER = 0, 1
 TUNE_INNER_GRID_CAP, TUNE_OUTER_GRID_CAP, TUNE_INNER_VARIANT, TUNE_PIPE_STAGES = 0, 1, 2, 3
-TUNE_CHUNK_MAJOR, TUNE_OUTER_SUB_ELEMS = 4, 5
+TUNE_CHUNK_MAJOR, TUNE_OUTER_SUB_ELEMS, TUNE_DDP_SUB_ELEMS = 4, 5, 6
 MAX_WORKERS = 64
 
 
@@ -53,6 +53,8 @@ def lib() -> C.CDLL:
     L.palsgd_init.argtypes = [C.POINTER(vp), C.POINTER(Config), C.c_size_t, u64p, C.POINTER(Buffers), vp]
     L.palsgd_inner_step.argtypes = [vp, C.c_double, C.c_double, vp]
     L.palsgd_pseudo_sync.argtypes = [vp, C.c_uint64, C.c_double, vp]
+    L.palsgd_ddp_step.argtypes = [vp, C.c_double, vp]
+    L.palsgd_ddp_step.restype = C.c_int
     L.palsgd_outer_sync.argtypes = [vp, vp]
     L.palsgd_step.argtypes = [vp, C.c_double, C.c_double, vp]
     L.palsgd_step_host.argtypes = [vp, C.POINTER(vp), C.c_double, C.c_double, C.POINTER(vp), u8p,
@@ -173,6 +175,9 @@ class Palsgd:
     # -- the C ABI, one method per entry point
     def inner_step(self, lr_t: float, eta_t: float, stream: int = 0) -> None:
         self._check(lib().palsgd_inner_step(self._ctx, lr_t, eta_t, C.c_void_p(stream)), "palsgd_inner_step")
+
+    def ddp_step(self, lr_t: float, stream: int = 0) -> None:
+        self._check(lib().palsgd_ddp_step(self._ctx, lr_t, C.c_void_p(stream)), "palsgd_ddp_step")
 
     def pseudo_sync(self, worker_mask: int, beta: float, stream: int = 0) -> None:
         self._check(lib().palsgd_pseudo_sync(self._ctx, worker_mask, beta, C.c_void_p(stream)), "palsgd_pseudo_sync")

@@ -48,6 +48,7 @@ struct palsgd_ctx {
     int chunk_major = 0;                          // work-item order of the register-path inner kernel
     uint32_t chunk_elems = kChunkElems;           // elements per chunk-table entry (fixed at init)
     uint32_t outer_sub_elems = kOuterSubElems;    // elements per work item of the outer kernel
+    uint32_t ddp_sub_elems = kDdpSubElems;        // elements per work item of the DDP warm-up kernel
     int sm_count = 0, smem_optin = 0;             // device attributes read at init
     std::string cuda_err;
 };
@@ -448,6 +449,43 @@ extern "C" int palsgd_inner_step(palsgd_ctx* ctx, double lr_t, double eta_t, voi
     return PALSGD_OK;
 }
 
+extern "C" int palsgd_ddp_step(palsgd_ctx* ctx, double lr_t, void* stream)
+{
+    if (!ctx) return PALSGD_EINVAL;
+    if (!finite_nonneg(lr_t)) return PALSGD_EINVAL;
+    const palsgd_config& c = ctx->cfg;
+    DdpArgs a{};
+    a.tb = ctx->tb;
+    a.beta1 = c.beta1;
+    a.beta2 = c.beta2;
+    a.lr = (float)lr_t;
+    a.b1 = (float)c.beta1;
+    a.b2 = (float)c.beta2;
+    a.omb1 = (float)(1.0 - c.beta1);
+    a.omb2 = (float)(1.0 - c.beta2);
+    a.eps = (float)c.eps;
+    a.decay = (float)(1.0 - lr_t * c.weight_decay);
+    a.mu = (float)c.momentum;
+    a.wd = (float)c.weight_decay;
+    a.Kf = (float)c.K;
+    a.sub_elems = ctx->ddp_sub_elems;
+    a.parts = (ctx->chunk_elems + a.sub_elems - 1) / a.sub_elems;
+    // with nothing to stream a one-CTA launch still advances the counters
+    const unsigned grid = grid_for((uint64_t)ctx->tb.n_chunks * a.parts, ctx->grid_cap_outer);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const bool adam = c.inner == PALSGD_INNER_ADAMW;
+    const bool bf = c.precision == PALSGD_PREC_BF16_MASTER;
+    int rc = launch_checked(ctx, [&] {
+        if (adam && !bf)       palsgd_ddp_kernel<0, 0><<<grid, kThreads, 0, s>>>(a);
+        else if (!adam && !bf) palsgd_ddp_kernel<1, 0><<<grid, kThreads, 0, s>>>(a);
+        else if (adam && bf)   palsgd_ddp_kernel<0, 1><<<grid, kThreads, 0, s>>>(a);
+        else                   palsgd_ddp_kernel<1, 1><<<grid, kThreads, 0, s>>>(a);
+    });
+    if (rc) return rc;
+    ctx->t += 1;
+    return PALSGD_OK;
+}
+
 extern "C" int palsgd_pseudo_sync(palsgd_ctx* ctx, uint64_t worker_mask, double beta, void* stream)
 {
     if (!ctx || !std::isfinite(beta)) return PALSGD_EINVAL;
@@ -618,6 +656,10 @@ extern "C" int palsgd_set_tuning(palsgd_ctx* ctx, int knob, int64_t value)
         case PALSGD_TUNE_OUTER_SUB_ELEMS:
             if (value < 1024 || value % 1024 != 0) return PALSGD_EINVAL;
             ctx->outer_sub_elems = (uint32_t)value;
+            return PALSGD_OK;
+        case PALSGD_TUNE_DDP_SUB_ELEMS:
+            if (value < 1024 || value % 1024 != 0) return PALSGD_EINVAL;
+            ctx->ddp_sub_elems = (uint32_t)value;
             return PALSGD_OK;
         default: return PALSGD_EINVAL;
     }

@@ -13,6 +13,7 @@ constexpr uint32_t kChunkElems  = 8192;    // default elements per chunk-table e
 constexpr uint32_t kStageElems  = 4096;    // stage size of the shared-memory-ring kernels
 constexpr uint32_t kOuterSubElems = 1024;  // default work item of the outer kernel: a slice of a chunk (small:
                                            // K+2 streams per element need many CTAs in flight)
+constexpr uint32_t kDdpSubElems = 2048;    // default work item of the DDP warm-up kernel (measured)
 constexpr uint32_t kSegVecFlag  = 0x80000000u;   // Chunk::seg bit: 16-byte vector path allowed
 
 // One work unit of the multi-tensor launch: `len` consecutive elements of
@@ -80,6 +81,18 @@ struct OuterArgs {
     int    nesterov;
     uint32_t sub_elems;    // elements per work item (a multiple of 4 * kThreads)
     uint32_t parts;        // work items per chunk = ceil(chunk_elems / sub_elems)
+};
+
+// DDP warm-up step: averaged gradient, one optimizer step taken on worker 0's state, written to all.
+struct DdpArgs {
+    Tables   tb;
+    double   beta1, beta2; // binary64 decay rates for the running products
+    float    lr;           // fl32(alpha_t): no 1/(1-p) rescaling in this phase
+    float    b1, b2, omb1, omb2, eps, decay;
+    float    mu, wd;
+    float    Kf;
+    uint32_t sub_elems;    // elements per work item (a multiple of 4 * kThreads)
+    uint32_t parts;        // work items per chunk
 };
 
 }  // namespace palsgd

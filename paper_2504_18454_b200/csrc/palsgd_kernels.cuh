@@ -652,6 +652,141 @@ palsgd_outer_kernel(const __grid_constant__ OuterArgs a)
     }
 }
 
+// ---------------------------------------------------------------- DDP warm-up step
+// Mini-batch phase that precedes Algorithm 1 (Sec. 3.3, Sec. 4.1): per element the K
+// gradients are summed in ascending k and divided by K, ONE optimizer step is taken on
+// worker 0's model and state with the plain step size alpha_t, and the result goes to
+// every slot and to the global model copy.  Reads 4K+12 bytes (2K+12 with bf16
+// gradients) and writes 12K+4 (14K+4) per parameter for AdamW: store-dominated, so the
+// work item is a small slice of a chunk, as in the outer kernel.
+
+template <int INNER, int PREC>
+__global__ void __launch_bounds__(kThreads)
+palsgd_ddp_kernel(const __grid_constant__ DdpArgs a)
+{
+    __shared__ float* s_x[kMaxWorkers];
+    __shared__ float* s_m[kMaxWorkers];
+    __shared__ float* s_v[kMaxWorkers];
+    __shared__ const void* s_g[kMaxWorkers];
+    __shared__ __nv_bfloat16* s_w[kMaxWorkers];
+    const Tables& tb = a.tb;
+    const uint32_t K = tb.K;
+    DevState* st = tb.st;
+    constexpr int B = 8;                                   // gradient loads issued together
+
+    // bias corrections for gradient step s_0 + 1 (all workers share worker 0's count in this phase)
+    const unsigned long long t = st->t;
+    AdamScalars as{a.b1, a.b2, a.omb1, a.omb2, 1.f, 1.f, a.decay, a.lr, a.eps};
+    if (INNER == 0) {
+        as.bc1 = (float)(1.0 - st->pow1[0] * a.beta1);
+        as.bc2 = (float)(1.0 - st->pow2[0] * a.beta2);
+    }
+    const SgdScalars ss{a.mu, a.wd, a.lr};
+
+    const uint64_t n_items = (uint64_t)tb.n_chunks * a.parts;
+    for (uint64_t item = blockIdx.x; item < n_items; item += gridDim.x) {
+        Chunk ch = tb.chunks[item / a.parts];
+        const uint32_t begin = (uint32_t)(item % a.parts) * a.sub_elems;
+        if (begin >= ch.len) continue;                                        // uniform over the CTA
+        ch.off += begin;
+        ch.len = min(ch.len - begin, a.sub_elems);
+        const uint32_t seg = ch.seg & ~kSegVecFlag;
+        __syncthreads();
+        if (threadIdx.x < K) {
+            const size_t pi = (size_t)threadIdx.x * tb.n_seg + seg;
+            s_x[threadIdx.x] = tb.xf[pi] + ch.off;
+            s_m[threadIdx.x] = tb.m[pi] + ch.off;
+            if (INNER == 0) s_v[threadIdx.x] = tb.v[pi] + ch.off;
+            if (PREC) { s_w[threadIdx.x] = tb.xw[pi] + ch.off;
+                        s_g[threadIdx.x] = static_cast<const __nv_bfloat16*>(tb.grad[pi]) + ch.off; }
+            else      { s_g[threadIdx.x] = static_cast<const float*>(tb.grad[pi]) + ch.off; }
+        }
+        __syncthreads();
+        float* xg = tb.global[seg] + ch.off;
+
+        uint32_t done = 0;
+        if (ch.seg & kSegVecFlag) {
+            const uint32_t n4 = ch.len >> 2;
+            for (uint32_t i = threadIdx.x; i < n4; i += kThreads) {
+                float4 X = __ldcs(reinterpret_cast<const float4*>(s_x[0]) + i);
+                float4 M = __ldcs(reinterpret_cast<const float4*>(s_m[0]) + i);
+                float4 V = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (INNER == 0) V = __ldcs(reinterpret_cast<const float4*>(s_v[0]) + i);
+                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                for (uint32_t k0 = 0; k0 < K; k0 += B) {
+                    float4 R[B];
+#pragma unroll
+                    for (int j = 0; j < B; ++j)
+                        if (k0 + j < K) {
+                            if (PREC) { const uint2 h = __ldcs(static_cast<const uint2*>(s_g[k0 + j]) + i);
+                                        float f[4]; unpack4(h, f); R[j] = make_float4(f[0], f[1], f[2], f[3]); }
+                            else      { R[j] = __ldcs(static_cast<const float4*>(s_g[k0 + j]) + i); }
+                        }
+#pragma unroll
+                    for (int j = 0; j < B; ++j)
+                        if (k0 + j < K) {
+                            if (k0 + j == 0) acc = R[j];
+                            else { acc.x = __fadd_rn(acc.x, R[j].x); acc.y = __fadd_rn(acc.y, R[j].y);
+                                   acc.z = __fadd_rn(acc.z, R[j].z); acc.w = __fadd_rn(acc.w, R[j].w); }
+                        }
+                }
+                float4 G;
+                G.x = __fdiv_rn(acc.x, a.Kf); G.y = __fdiv_rn(acc.y, a.Kf);
+                G.z = __fdiv_rn(acc.z, a.Kf); G.w = __fdiv_rn(acc.w, a.Kf);
+                if (INNER == 0) { PALSGD_FOR4(adamw_elem(compv(G, c), comp(X, c), comp(M, c), comp(V, c), as)) }
+                else            { PALSGD_FOR4(sgdm_elem(compv(G, c), comp(X, c), comp(M, c), ss)) }
+                __stcs(reinterpret_cast<float4*>(xg) + i, X);
+                for (uint32_t k = 0; k < K; ++k) {
+                    __stcs(reinterpret_cast<float4*>(s_x[k]) + i, X);
+                    __stcs(reinterpret_cast<float4*>(s_m[k]) + i, M);
+                    if (INNER == 0) __stcs(reinterpret_cast<float4*>(s_v[k]) + i, V);
+                }
+                if (PREC) {
+                    const uint2 h = pack4(X);
+                    for (uint32_t k = 0; k < K; ++k) __stcs(reinterpret_cast<uint2*>(s_w[k]) + i, h);
+                }
+            }
+            done = n4 << 2;
+        }
+        for (uint32_t i = done + threadIdx.x; i < ch.len; i += kThreads) {
+            float sum = 0.f;
+            for (uint32_t k = 0; k < K; ++k) {
+                const float gk = PREC ? __bfloat162float(static_cast<const __nv_bfloat16*>(s_g[k])[i])
+                                      : static_cast<const float*>(s_g[k])[i];
+                sum = k == 0 ? gk : __fadd_rn(sum, gk);
+            }
+            const float g = __fdiv_rn(sum, a.Kf);
+            float xi = s_x[0][i], mi = s_m[0][i], vi = 0.f;
+            if (INNER == 0) { vi = s_v[0][i]; adamw_elem(g, xi, mi, vi, as); }
+            else            { sgdm_elem(g, xi, mi, ss); }
+            xg[i] = xi;
+            for (uint32_t k = 0; k < K; ++k) {
+                s_x[k][i] = xi; s_m[k][i] = mi;
+                if (INNER == 0) s_v[k][i] = vi;
+                if (PREC) s_w[k][i] = __float2bfloat16_rn(xi);
+            }
+        }
+    }
+
+    // ---- counter tick by the last CTA (all state reads above precede the atomic)
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        const unsigned int prev = atomicAdd(&st->done, 1u);
+        if (prev == gridDim.x - 1) {
+            const unsigned long long s0 = st->s[0] + 1;
+            const double p1 = INNER == 0 ? st->pow1[0] * a.beta1 : st->pow1[0];
+            const double p2 = INNER == 0 ? st->pow2[0] * a.beta2 : st->pow2[0];
+            for (uint32_t k = 0; k < K; ++k) {
+                st->s[k] = s0; st->pow1[k] = p1; st->pow2[k] = p2; st->last_b[k] = 0;
+            }
+            st->t = t + 1;
+            st->done = 0;
+            __threadfence();
+        }
+    }
+}
+
 // ---------------------------------------------------------------- set-up
 // x_g <- fixed-order mean of the slots, u <- 0, m, v <- 0, bf16 working <- RNE(master).
 template <int PREC>

@@ -77,6 +77,18 @@ def _child(args) -> None:
         per = (10 if cfg.precision == 1 else 8) * cfg.K + 16
         return per * cfg.P / (e0.elapsed_time(e1) / reps) / 1e6
 
+    def time_ddp(reps=8):
+        for _ in range(2):
+            ctx.ddp_step(cfg.lr, stream)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            ctx.ddp_step(cfg.lr, stream)
+        e1.record()
+        torch.cuda.synchronize()
+        per = (16 if cfg.inner == 0 else 12) * (cfg.K + 1)      # both precisions: see include/palsgd.h
+        return per * cfg.P / (e0.elapsed_time(e1) / reps) / 1e6
+
     for v in args.variants:
         ctx.set_tuning(P.TUNE_INNER_VARIANT, v)
         r = sorted(time_inner(args.steps) for _ in range(3))
@@ -85,6 +97,9 @@ def _child(args) -> None:
         ctx.set_tuning(P.TUNE_OUTER_SUB_ELEMS, sub)
         r = sorted(time_outer() for _ in range(3))
         print(f"{cfg.name} chunk={chunk} outer slice={sub}: {r[1]:.0f} GB/s (runs {r[0]:.0f}..{r[2]:.0f})", flush=True)
+        ctx.set_tuning(P.TUNE_DDP_SUB_ELEMS, sub)
+        r = sorted(time_ddp() for _ in range(3))
+        print(f"{cfg.name} chunk={chunk} ddp slice={sub}: {r[1]:.0f} GB/s (runs {r[0]:.0f}..{r[2]:.0f})", flush=True)
     ctx.destroy()
 
 

@@ -133,6 +133,9 @@ class GpuRun:
     def outer_sync(self):
         self.lib.outer_sync(self.stream)
 
+    def ddp_step(self, lr):
+        self.lib.ddp_step(lr, self.stream)
+
     def pseudo_sync(self, mask, beta):
         self.lib.pseudo_sync(mask, beta, self.stream)
 

@@ -55,7 +55,8 @@ def test_model_shaped_lists_every_element_short_schedule(name, layout):
     assert gpu.guards_intact()
 
 
-def _full_size_sampled(cfg, n_random, T=None):
+def _full_size_sampled(cfg, n_random, T=None, n_ddp=0):
+    """n_ddp: that many leading steps are DDP warm-up steps."""
     T = cfg.T if T is None else T
     dev = torch.device("cuda:0")
     tensors = cfg.tensors
@@ -74,8 +75,12 @@ def _full_size_sampled(cfg, n_random, T=None):
             grad_rows[k].copy_(r)                     # rounds to bf16 in mixed-precision mode
         gs = grad_rows[:, idx_d].contiguous()
         gs = gs.view(torch.int16).cpu().numpy().view(np.uint16) if cfg.precision == 1 else gs.cpu().numpy()
-        gpu.step(cfg.lr, cfg.eta)
-        orc.step(gs, cfg.lr, cfg.eta)
+        if t < n_ddp:
+            gpu.ddp_step(cfg.lr)
+            orc.ddp_step(gs, cfg.lr)
+        else:
+            gpu.step(cfg.lr, cfg.eta)
+            orc.step(gs, cfg.lr, cfg.eta)
     torch.cuda.synchronize()
     c = gpu.counters()
     assert c["t"] == orc.t == T and c["n_outer"] == orc.n_outer
@@ -116,3 +121,9 @@ def test_c3_gptneo125m_bf16_full_size_full_schedule_sampled():
 def test_sweep_corner_k32_large_flat_buffer_sampled():
     cfg = next(c for c in W.sweep_points() if c.K == 32 and c.P == 1 << 24 and c.p == 0.5 and c.H == 16)
     _full_size_sampled(cfg, 1 << 14, T=32)
+
+
+@pytest.mark.parametrize("name", ["c2_resnet50", "c3_gptneo125m_bf16"])
+def test_ddp_warm_up_then_palsgd_full_size_sampled(name):
+    cfg = W.get_config(name).with_(H=4)
+    _full_size_sampled(cfg, 1 << 14, T=12, n_ddp=6)
