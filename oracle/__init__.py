@@ -42,6 +42,12 @@ def lib() -> C.CDLL:
         L.palsgd_oracle_bf16_from_f32.restype = C.c_uint16
         L.palsgd_oracle_bf16_from_f64.argtypes = [C.c_double]
         L.palsgd_oracle_bf16_from_f64.restype = C.c_uint16
+        for name, ct in (("f32", C.c_float), ("f64", C.c_double), ("bf16", C.c_uint16)):
+            f = getattr(L, f"palsgd_oracle_sumsq_{name}")
+            f.argtypes = [C.POINTER(ct), C.c_uint64]
+            f.restype = C.c_double
+        L.palsgd_oracle_clip_coef.argtypes = [C.c_double, C.c_double]
+        L.palsgd_oracle_clip_coef.restype = C.c_double
         L.palsgd_oracle_set_threads.argtypes = [C.c_int]
         L.palsgd_oracle_set_threads.restype = None
         L.palsgd_oracle_get_threads.argtypes = []
@@ -82,6 +88,19 @@ def bf16_to_f32(h: int) -> float:
     return float(lib().palsgd_oracle_bf16_to_f32(int(h)))
 
 
+def sumsq(g: np.ndarray) -> float:
+    """Exact sum of squares of a float32 / float64 array, or of bf16 bit patterns (uint16),
+    rounded once to binary64."""
+    g = np.ascontiguousarray(g).reshape(-1)
+    name, ct = {np.dtype(np.float32): ("f32", C.c_float), np.dtype(np.float64): ("f64", C.c_double),
+                np.dtype(np.uint16): ("bf16", C.c_uint16)}[g.dtype]
+    return float(getattr(lib(), f"palsgd_oracle_sumsq_{name}")(g.ctypes.data_as(C.POINTER(ct)), g.size))
+
+
+def clip_coef(sumsq_: float, max_norm: float) -> float:
+    return float(lib().palsgd_oracle_clip_coef(float(sumsq_), float(max_norm)))
+
+
 def set_threads(n: int) -> None:
     lib().palsgd_oracle_set_threads(int(n))
 
@@ -106,6 +125,8 @@ def _state_struct(real):
             ("t", C.c_uint64), ("s", C.POINTER(C.c_uint64)), ("n_outer", C.c_uint64),
             ("pow1", C.POINTER(C.c_double)), ("pow2", C.POINTER(C.c_double)),
             ("last_b", C.POINTER(C.c_uint8)),
+            ("max_grad_norm", C.c_double), ("forced_sumsq", C.POINTER(C.c_double)),
+            ("sumsq", C.POINTER(C.c_double)), ("clipc", C.POINTER(C.c_double)),
         ]
 
     return State
@@ -127,7 +148,7 @@ class Oracle:
                  weight_decay: float = 0.01, momentum: float = 0.0,
                  outer_lr: float = 0.7, outer_momentum: float = 0.9,
                  outer_nesterov: bool = True, seed: int = 0, precision: int = 0,
-                 dtype: str = "f32"):
+                 max_grad_norm: float = 0.0, dtype: str = "f32"):
         x0 = np.asarray(x0)
         assert x0.ndim == 2 and x0.shape[0] == K, x0.shape
         self.dtype = dtype
@@ -143,6 +164,9 @@ class Oracle:
         self.pow1 = np.ones(self.K, dtype=np.float64)
         self.pow2 = np.ones(self.K, dtype=np.float64)
         self.last_b = np.zeros(self.K, dtype=np.uint8)
+        self.sumsq = np.zeros(self.K, dtype=np.float64)
+        self.clipc = np.ones(self.K, dtype=np.float64)
+        self._forced_sumsq = None
         S = _STATE[dtype]
         p_ = lambda a, t: a.ctypes.data_as(C.POINTER(t))
         self._st = S(
@@ -155,7 +179,9 @@ class Oracle:
             xw=p_(self.xw, C.c_uint16) if self.xw is not None else None,
             t=0, s=p_(self.s, C.c_uint64), n_outer=0,
             pow1=p_(self.pow1, C.c_double), pow2=p_(self.pow2, C.c_double),
-            last_b=p_(self.last_b, C.c_uint8))
+            last_b=p_(self.last_b, C.c_uint8),
+            max_grad_norm=float(max_grad_norm), forced_sumsq=None,
+            sumsq=p_(self.sumsq, C.c_double), clipc=p_(self.clipc, C.c_double))
         L = lib()
         sfx = dtype
         self._init = getattr(L, f"palsgd_oracle_init_{sfx}")
@@ -183,6 +209,21 @@ class Oracle:
     @property
     def n_outer(self) -> int:
         return int(self._st.n_outer)
+
+    # gradient clipping ---------------------------------------------------
+    def set_grad_clip(self, max_norm: float) -> None:
+        self._st.max_grad_norm = float(max_norm)
+
+    def force_sumsq(self, sumsq_per_worker) -> None:
+        """Use these K sums of squares in the following steps instead of computing them from the
+        gradients passed in (for replays of a sample of a large run); None switches back."""
+        if sumsq_per_worker is None:
+            self._forced_sumsq = None
+            self._st.forced_sumsq = None
+        else:
+            self._forced_sumsq = np.ascontiguousarray(sumsq_per_worker, dtype=np.float64)
+            assert self._forced_sumsq.shape == (self.K,)
+            self._st.forced_sumsq = self._forced_sumsq.ctypes.data_as(C.POINTER(C.c_double))
 
     # steps ---------------------------------------------------------------
     def _grads_ptr(self, grads: np.ndarray):

@@ -21,6 +21,14 @@
 #include <math.h>
 #include <stdint.h>
 #include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+static int oracle_thread_id(void)    { return omp_get_thread_num(); }
+static int oracle_thread_count(void) { return omp_get_num_threads(); }
+#else
+static int oracle_thread_id(void)    { return 0; }
+static int oracle_thread_count(void) { return 1; }
+#endif
 
 /* ---- Philox4x32-10 ------------------------------------------------------ */
 
@@ -125,9 +133,61 @@ uint16_t palsgd_oracle_bf16_from_f64(double d)
     return (uint16_t)(sign | (uint16_t)(u >> 16));
 }
 
+/* ---- global gradient norm ------------------------------------------------- */
+
+/* The sum of squares behind a global-norm gradient clip, defined here as the
+ * EXACT sum  sum_i g_i^2  rounded once to binary64.  It is realised with
+ * binary128 arithmetic: every square of a binary32/binary64 value is exact in
+ * binary128, and the accumulated rounding error of n additions (n * 2^-113
+ * relative) is far below half a unit of binary64, so the result is the correctly
+ * rounded exact sum except with negligible probability.  Because the sum is
+ * exact, the order of the terms does not matter; the index range is split into
+ * one contiguous block per thread and the block sums are added in block order.
+ * Not re-entrant (one static table of block sums).                             */
+#define SUMSQ_MAX_THREADS 1024
+#define SUMSQ_BODY(LOAD)                                                        \
+    static __float128 part[SUMSQ_MAX_THREADS];                                  \
+    int used = 1;                                                               \
+    _Pragma("omp parallel")                                                     \
+    {                                                                           \
+        int me = 0, nt = 1;                                                     \
+        me = oracle_thread_id(); nt = oracle_thread_count();                    \
+        if (nt > SUMSQ_MAX_THREADS) nt = SUMSQ_MAX_THREADS;                     \
+        if (me == 0) used = nt;                                                 \
+        if (me < nt) {                                                          \
+            /* thread `me` sums the contiguous block [lo, hi) */                \
+            uint64_t lo = n / (uint64_t)nt * (uint64_t)me;                      \
+            uint64_t hi = me == nt - 1 ? n : n / (uint64_t)nt * (uint64_t)(me + 1); \
+            __float128 acc = 0;                                                 \
+            for (uint64_t i = lo; i < hi; ++i) {                                \
+                __float128 x = (__float128)(LOAD);                              \
+                acc += x * x;                                                   \
+            }                                                                   \
+            part[me] = acc;                                                     \
+        }                                                                       \
+    }                                                                           \
+    __float128 total = 0;                                                       \
+    for (int j = 0; j < used; ++j) total += part[j];                            \
+    return (double)total;
+
+double palsgd_oracle_sumsq_f32(const float *g, uint64_t n)     { SUMSQ_BODY(g[i]) }
+double palsgd_oracle_sumsq_f64(const double *g, uint64_t n)    { SUMSQ_BODY(g[i]) }
+double palsgd_oracle_sumsq_bf16(const uint16_t *g, uint64_t n) { SUMSQ_BODY(palsgd_oracle_bf16_to_f32(g[i])) }
+
+/* Clip coefficient of a global-norm clip with threshold max_norm, in the
+ * convention of the software the paper ran (PyTorch's clip_grad_norm_; the paper
+ * only says that clipping was enabled, Appendix B):
+ *     norm = sqrt(sumsq);  c = max_norm / (norm + 1e-6);  c = min(c, 1),
+ * all in binary64.  The gradient is then multiplied by c.                       */
+double palsgd_oracle_clip_coef(double sumsq, double max_norm)
+{
+    double norm = sqrt(sumsq);
+    double c = max_norm / (norm + 1e-6);
+    return c < 1.0 ? c : 1.0;
+}
+
 /* ---- thread count of the element loops (timing harness only) -------------- */
 #ifdef _OPENMP
-#include <omp.h>
 void palsgd_oracle_set_threads(int n) { if (n > 0) omp_set_num_threads(n); }
 int  palsgd_oracle_get_threads(void)  { return omp_get_max_threads(); }
 #else

@@ -29,6 +29,7 @@
 #include <math.h>
 #include <stddef.h>
 #include <stdint.h>
+#include <stdlib.h>
 
 #ifndef REAL
 #error "compile with -DREAL=float|double -DSUFFIX=f32|f64"
@@ -41,6 +42,10 @@ int      palsgd_oracle_decision(uint64_t seed, uint64_t t, uint32_t k, double p)
 float    palsgd_oracle_bf16_to_f32(uint16_t h);
 uint16_t palsgd_oracle_bf16_from_f32(float f);
 uint16_t palsgd_oracle_bf16_from_f64(double d);
+double   palsgd_oracle_sumsq_f32(const float *g, uint64_t n);
+double   palsgd_oracle_sumsq_f64(const double *g, uint64_t n);
+double   palsgd_oracle_sumsq_bf16(const uint16_t *g, uint64_t n);
+double   palsgd_oracle_clip_coef(double sumsq, double max_norm);
 
 typedef struct {
     /* Algorithm 1's data line */
@@ -66,6 +71,12 @@ typedef struct {
     uint64_t  n_outer;       /* outer syncs performed                              */
     double   *pow1, *pow2;   /* [K] beta1^s_k, beta2^s_k (running products)        */
     uint8_t  *last_b;        /* [K] decisions of the latest step                   */
+    /* global-norm gradient clipping (Appendix B: "gradient clipping enabled") */
+    double    max_grad_norm; /* threshold; 0 = no clipping                         */
+    const double *forced_sumsq; /* NULL, or [K] sums of squares to use instead of
+                                computing them (sampled replays of a large run)   */
+    double   *sumsq;         /* [K] sum of squares of the latest gradients seen    */
+    double   *clipc;         /* [K] coefficient the latest gradient was scaled by  */
 } FN(state);
 
 static uint16_t to_bf16(REAL a)
@@ -126,7 +137,7 @@ static void pull_worker(FN(state) *st, uint32_t k, REAL beta)
 
 /* InnerOPT = AdamW with step size lr (Eq. (1): lr = alpha_t / (1 - p)). */
 static void adamw_worker(FN(state) *st, uint32_t k, const float *g32, const uint16_t *g16,
-                         double lr_d)
+                         double lr_d, REAL clip)
 {
     const size_t P = st->P;
     REAL *x = st->x + (size_t)k * P, *m = st->m + (size_t)k * P, *v = st->v + (size_t)k * P;
@@ -143,6 +154,7 @@ static void adamw_worker(FN(state) *st, uint32_t k, const float *g32, const uint
     #pragma omp parallel for schedule(static)
     for (int64_t i = 0; i < (int64_t)P; ++i) {
         REAL g = g32 ? (REAL)g32[i] : (REAL)palsgd_oracle_bf16_to_f32(g16[i]);
+        g = g * clip;                                   /* clipped gradient (clip = 1: unchanged) */
         REAL mi = b1 * m[i] + omb1 * g;
         REAL vi = b2 * v[i] + omb2 * (g * g);
         REAL mhat = mi / bc1;
@@ -158,7 +170,7 @@ static void adamw_worker(FN(state) *st, uint32_t k, const float *g32, const uint
 /* InnerOPT = momentum SGD with step size lr; L2 decay added to the gradient,
  * buffer starts at zero, no dampening, no Nesterov. */
 static void sgdm_worker(FN(state) *st, uint32_t k, const float *g32, const uint16_t *g16,
-                        double lr_d)
+                        double lr_d, REAL clip)
 {
     const size_t P = st->P;
     REAL *x = st->x + (size_t)k * P, *buf = st->m + (size_t)k * P;
@@ -167,6 +179,7 @@ static void sgdm_worker(FN(state) *st, uint32_t k, const float *g32, const uint1
     #pragma omp parallel for schedule(static)
     for (int64_t i = 0; i < (int64_t)P; ++i) {
         REAL g = g32 ? (REAL)g32[i] : (REAL)palsgd_oracle_bf16_to_f32(g16[i]);
+        g = g * clip;
         REAL gp = g + wd * x[i];
         REAL b = mu * buf[i] + gp;
         buf[i] = b;
@@ -203,8 +216,17 @@ int FN(inner_step)(FN(state) *st, const void *grads, double alpha_t, double eta_
             double lr_d = alpha_t / (1.0 - st->p);
             const float *g32 = st->precision == 0 ? (const float *)grads + (size_t)k * st->P : NULL;
             const uint16_t *g16 = st->precision == 1 ? (const uint16_t *)grads + (size_t)k * st->P : NULL;
-            if (st->inner == 0) adamw_worker(st, k, g32, g16, lr_d);
-            else                sgdm_worker(st, k, g32, g16, lr_d);
+            /* clip this worker's gradient to global norm max_grad_norm before InnerOPT sees it */
+            REAL clip = (REAL)1;
+            if (st->max_grad_norm > 0.0) {
+                double ss = st->forced_sumsq ? st->forced_sumsq[k]
+                          : g32 ? palsgd_oracle_sumsq_f32(g32, st->P) : palsgd_oracle_sumsq_bf16(g16, st->P);
+                double c = palsgd_oracle_clip_coef(ss, st->max_grad_norm);
+                st->sumsq[k] = ss; st->clipc[k] = c;
+                clip = (REAL)c;
+            }
+            if (st->inner == 0) adamw_worker(st, k, g32, g16, lr_d, clip);
+            else                sgdm_worker(st, k, g32, g16, lr_d, clip);
         }
     }
     st->t += 1;
@@ -278,13 +300,31 @@ void FN(ddp_step)(FN(state) *st, const void *grads, double alpha_t)
     const REAL eps   = (REAL)st->eps;
     const REAL mu    = (REAL)st->momentum, wd = (REAL)st->weight_decay;
 
+    /* averaged gradient */
+    REAL *gbar = (REAL *)malloc((P ? P : 1) * sizeof(REAL));
+    if (!gbar) return;
     #pragma omp parallel for schedule(static)
     for (int64_t i = 0; i < (int64_t)P; ++i) {
         REAL sum = g32 ? (REAL)g32[i] : (REAL)palsgd_oracle_bf16_to_f32(g16[i]);
         for (uint32_t k = 1; k < K; ++k)
             sum = sum + (g32 ? (REAL)g32[(size_t)k * P + i]
                              : (REAL)palsgd_oracle_bf16_to_f32(g16[(size_t)k * P + i]));
-        REAL g = sum / (REAL)K;
+        gbar[i] = sum / (REAL)K;
+    }
+    /* in this phase the clip applies to the averaged gradient */
+    REAL clip = (REAL)1;
+    if (st->max_grad_norm > 0.0) {
+        double ssq = st->forced_sumsq ? st->forced_sumsq[0]
+                   : sizeof(REAL) == 4 ? palsgd_oracle_sumsq_f32((const float *)(const void *)gbar, P)
+                                       : palsgd_oracle_sumsq_f64((const double *)(const void *)gbar, P);
+        double c = palsgd_oracle_clip_coef(ssq, st->max_grad_norm);
+        for (uint32_t k = 0; k < K; ++k) { st->sumsq[k] = ssq; st->clipc[k] = c; }
+        clip = (REAL)c;
+    }
+
+    #pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < (int64_t)P; ++i) {
+        REAL g = gbar[i] * clip;
         REAL xi;
         if (st->inner == 0) {
             REAL mi = b1 * m[i] + omb1 * g;
@@ -304,6 +344,7 @@ void FN(ddp_step)(FN(state) *st, const void *grads, double alpha_t)
         for (uint32_t k = 0; k < K; ++k) x[(size_t)k * P + i] = xi;
         st->xg[i] = xi;
     }
+    free(gbar);
     for (uint32_t k = 0; k < K; ++k) {
         st->s[k] = st->s[0]; st->pow1[k] = st->pow1[0]; st->pow2[k] = st->pow2[0];
         st->last_b[k] = 0;
