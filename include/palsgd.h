@@ -199,6 +199,28 @@ int palsgd_get_counters(palsgd_ctx* ctx, uint64_t* t, uint64_t* s_k, uint64_t* n
 int palsgd_set_counters(palsgd_ctx* ctx, uint64_t t, const uint64_t* s_k, uint64_t n_outer,
                         void* stream);
 
+/*
+ * Global-norm gradient clipping (Appendix B trains GPT-Neo "with gradient clipping
+ * enabled" and gives no threshold, so it is a parameter here).  max_norm > 0 turns it
+ * on for the following palsgd_inner_step / palsgd_step / palsgd_ddp_step calls,
+ * 0 turns it off (the default).  Convention of the software the paper ran
+ * (clip_grad_norm_), per worker k that takes a gradient step:
+ *   sumsq_k = the exact sum over the worker's WHOLE gradient (all tensors) of g^2,
+ *             rounded once to binary64
+ *   c_k = fl32(min(1, max_norm / (sqrt(sumsq_k) + 1e-6)))     (binary64, rounded once)
+ *   g <- g * c_k (one binary32 multiplication) before InnerOPT sees it.
+ * Workers that pull in a step have no norm taken.  In the DDP phase the one norm is
+ * that of the averaged gradient gbar.  Costs one extra kernel launch per step that
+ * reads every gradient once more.
+ * Errors: EINVAL (NULL ctx, negative or non-finite max_norm).
+ */
+int palsgd_set_grad_clip(palsgd_ctx* ctx, double max_norm);
+
+/* The sums of squares and clip coefficients of the latest clipped step (K each; either
+ * pointer may be NULL; entries of workers that pulled keep their previous values;
+ * before the first clipped step: 0 and 1).  SYNCHRONISES the stream. */
+int palsgd_get_grad_norms(palsgd_ctx* ctx, double* sumsq, float* clip, void* stream);
+
 /* Number of kernels this context has launched so far (host-side count). */
 int palsgd_get_launch_count(palsgd_ctx* ctx, uint64_t* n_launches);
 

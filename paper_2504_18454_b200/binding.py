@@ -55,6 +55,10 @@ def lib() -> C.CDLL:
     L.palsgd_pseudo_sync.argtypes = [vp, C.c_uint64, C.c_double, vp]
     L.palsgd_ddp_step.argtypes = [vp, C.c_double, vp]
     L.palsgd_ddp_step.restype = C.c_int
+    L.palsgd_set_grad_clip.argtypes = [vp, C.c_double]
+    L.palsgd_set_grad_clip.restype = C.c_int
+    L.palsgd_get_grad_norms.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_float), vp]
+    L.palsgd_get_grad_norms.restype = C.c_int
     L.palsgd_outer_sync.argtypes = [vp, vp]
     L.palsgd_step.argtypes = [vp, C.c_double, C.c_double, vp]
     L.palsgd_step_host.argtypes = [vp, C.POINTER(vp), C.c_double, C.c_double, C.POINTER(vp), u8p,
@@ -215,6 +219,14 @@ class Palsgd:
     def set_counters(self, t: int, s: Sequence[int], n_outer: int, stream: int = 0) -> None:
         arr = (C.c_uint64 * self.K)(*[int(x) for x in s])
         self._check(lib().palsgd_set_counters(self._ctx, t, arr, n_outer, C.c_void_p(stream)), "palsgd_set_counters")
+
+    def set_grad_clip(self, max_norm: float) -> None:
+        self._check(lib().palsgd_set_grad_clip(self._ctx, max_norm), "palsgd_set_grad_clip")
+
+    def get_grad_norms(self, stream: int = 0):
+        ss, cl = (C.c_double * self.K)(), (C.c_float * self.K)()
+        self._check(lib().palsgd_get_grad_norms(self._ctx, ss, cl, C.c_void_p(stream)), "palsgd_get_grad_norms")
+        return list(ss), list(cl)
 
     def get_launch_count(self) -> int:
         n = C.c_uint64(0)

@@ -17,6 +17,7 @@
 #include <vector>
 
 #include "palsgd_kernels.cuh"
+#include "palsgd_norm.cuh"
 #include "palsgd_pipe.cuh"
 
 using namespace palsgd;
@@ -49,6 +50,7 @@ struct palsgd_ctx {
     uint32_t chunk_elems = kChunkElems;           // elements per chunk-table entry (fixed at init)
     uint32_t outer_sub_elems = kOuterSubElems;    // elements per work item of the outer kernel
     uint32_t ddp_sub_elems = kDdpSubElems;        // elements per work item of the DDP warm-up kernel
+    double max_grad_norm = 0.0;                   // global-norm clip threshold, 0 = off
     int sm_count = 0, smem_optin = 0;             // device attributes read at init
     std::string cuda_err;
 };
@@ -204,9 +206,34 @@ int launch_inner_pipe_nc(palsgd_ctx* ctx, int variant, const InnerArgs& a, cudaS
     return launch_inner_pipe<INNER, PREC, 0>(ctx, a, s);
 }
 
+// Norm pass of the gradient clip: per-worker norms (ddp = false) or the norm of the averaged gradient.
+int launch_gradnorm(palsgd_ctx* ctx, bool ddp, cudaStream_t s)
+{
+    NormArgs a{};
+    a.tb = ctx->tb;
+    a.seed = ctx->cfg.seed;
+    a.thr = ctx->thr;
+    a.max_norm = ctx->max_grad_norm;
+    a.Kf = (float)ctx->cfg.K;
+    a.ddp = ddp ? 1u : 0u;
+    // chunks per work item: up to 8 (4 for the K-stream averaged form), fewer while that would leave
+    // under ~2048 items; fixed by the problem, so results never depend on the device or on tuning knobs
+    const uint32_t kitems = ddp ? 1u : ctx->cfg.K;
+    const uint64_t items1 = (uint64_t)ctx->tb.n_chunks * kitems;
+    a.group = (uint32_t)std::min<uint64_t>(ddp ? 4 : 8, std::max<uint64_t>(1, items1 / 2048));
+    const uint64_t n_groups = (ctx->tb.n_chunks + a.group - 1) / a.group;
+    const unsigned grid = grid_for(n_groups * kitems, ctx->grid_cap_inner);
+    const bool bf = ctx->cfg.precision == PALSGD_PREC_BF16_MASTER;
+    return launch_checked(ctx, [&] {
+        if (bf) palsgd_gradnorm_kernel<1><<<grid, kThreads, 0, s>>>(a);
+        else    palsgd_gradnorm_kernel<0><<<grid, kThreads, 0, s>>>(a);
+    });
+}
+
 int launch_inner(palsgd_ctx* ctx, const InnerArgs& a, cudaStream_t s)
 {
-    if (ctx->inner_variant >= 10 && ctx->inner_variant <= 12 && ctx->tb.n_full > 0 &&
+    // the shared-memory-ring forms do not carry the clip coefficient: clipped steps take the register path
+    if (!a.clip_on && ctx->inner_variant >= 10 && ctx->inner_variant <= 12 && ctx->tb.n_full > 0 &&
         ctx->chunk_elems % kStageElems == 0) {
         const bool adam_ = ctx->cfg.inner == PALSGD_INNER_ADAMW;
         const bool bf_ = ctx->cfg.precision == PALSGD_PREC_BF16_MASTER;
@@ -341,10 +368,11 @@ extern "C" int palsgd_init(palsgd_ctx** out, const palsgd_config* cfg, size_t n_
     size_t off_state = 0;
     size_t off_chunks = round_up(sizeof(DevState), 256);
     size_t off_tabs = round_up(off_chunks + chunks.size() * sizeof(Chunk), 256);
-    const size_t total = off_tabs + 5 * round_up(per_slot, 256) + 2 * round_up(per_seg, 256) + 256;
+    const size_t off_norm = off_tabs + 5 * round_up(per_slot, 256) + 2 * round_up(per_seg, 256) + 256;
+    const size_t total = off_norm + round_up(chunks.size() * K * sizeof(double2), 256) + 256;
     std::vector<char> host(total, 0);
     DevState hs{};
-    for (uint32_t k = 0; k < kMaxWorkers; ++k) { hs.pow1[k] = 1.0; hs.pow2[k] = 1.0; }
+    for (uint32_t k = 0; k < kMaxWorkers; ++k) { hs.pow1[k] = 1.0; hs.pow2[k] = 1.0; hs.clip[k] = 1.f; }
     std::memcpy(host.data() + off_state, &hs, sizeof(hs));
     if (!chunks.empty()) std::memcpy(host.data() + off_chunks, chunks.data(), chunks.size() * sizeof(Chunk));
 
@@ -399,6 +427,7 @@ extern "C" int palsgd_init(palsgd_ctx** out, const palsgd_config* cfg, size_t n_
     tb.outer_mom = static_cast<float* const*>(fill_seg_table(bufs->outer_mom));
     tb.xf = static_cast<float* const*>(bf ? t_master : t_param);
     tb.xw = bf ? static_cast<__nv_bfloat16* const*>(t_param) : nullptr;
+    tb.norm_part = reinterpret_cast<double2*>(d + off_norm);
 
     cudaError_t e = cudaMemcpyAsync(ctx->d_blob, host.data(), total, cudaMemcpyHostToDevice, s);
     if (e == cudaSuccess) e = cudaStreamSynchronize(s);      // `host` is pageable and dies with this scope
@@ -443,7 +472,11 @@ extern "C" int palsgd_inner_step(palsgd_ctx* ctx, double lr_t, double eta_t, voi
     a.mu = (float)c.momentum;
     a.wd = (float)c.weight_decay;
     a.chunk_major = (uint32_t)ctx->chunk_major;
-    int rc = launch_inner(ctx, a, static_cast<cudaStream_t>(stream));
+    // clipped gradients: one norm pass first (not needed when every worker pulls)
+    a.clip_on = (ctx->max_grad_norm > 0.0 && c.p < 1.0) ? 1u : 0u;
+    int rc = PALSGD_OK;
+    if (a.clip_on) { rc = launch_gradnorm(ctx, false, static_cast<cudaStream_t>(stream)); if (rc) return rc; }
+    rc = launch_inner(ctx, a, static_cast<cudaStream_t>(stream));
     if (rc) return rc;
     ctx->t += 1;
     return PALSGD_OK;
@@ -475,7 +508,10 @@ extern "C" int palsgd_ddp_step(palsgd_ctx* ctx, double lr_t, void* stream)
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const bool adam = c.inner == PALSGD_INNER_ADAMW;
     const bool bf = c.precision == PALSGD_PREC_BF16_MASTER;
-    int rc = launch_checked(ctx, [&] {
+    a.clip_on = ctx->max_grad_norm > 0.0 ? 1u : 0u;
+    int rc = PALSGD_OK;
+    if (a.clip_on) { rc = launch_gradnorm(ctx, true, s); if (rc) return rc; }
+    rc = launch_checked(ctx, [&] {
         if (adam && !bf)       palsgd_ddp_kernel<0, 0><<<grid, kThreads, 0, s>>>(a);
         else if (!adam && !bf) palsgd_ddp_kernel<1, 0><<<grid, kThreads, 0, s>>>(a);
         else if (adam && bf)   palsgd_ddp_kernel<0, 1><<<grid, kThreads, 0, s>>>(a);
@@ -620,7 +656,7 @@ extern "C" int palsgd_set_counters(palsgd_ctx* ctx, uint64_t t, const uint64_t* 
     DevState hs{};
     hs.t = t;
     for (uint32_t k = 0; k < kMaxWorkers; ++k) {
-        hs.pow1[k] = 1.0; hs.pow2[k] = 1.0;
+        hs.pow1[k] = 1.0; hs.pow2[k] = 1.0; hs.clip[k] = 1.f;
         if (k < ctx->cfg.K) {
             hs.s[k] = s_k[k];
             for (uint64_t i = 0; i < s_k[k]; ++i) {      // the same running products the kernels form
@@ -634,6 +670,27 @@ extern "C" int palsgd_set_counters(palsgd_ctx* ctx, uint64_t t, const uint64_t* 
     PALSGD_CUDA(ctx, cudaStreamSynchronize(s));          // hs lives on this stack frame
     ctx->t = t;
     ctx->n_outer = n_outer;
+    return PALSGD_OK;
+}
+
+extern "C" int palsgd_set_grad_clip(palsgd_ctx* ctx, double max_norm)
+{
+    if (!ctx || !(max_norm >= 0.0) || !std::isfinite(max_norm)) return PALSGD_EINVAL;
+    ctx->max_grad_norm = max_norm;
+    return PALSGD_OK;
+}
+
+extern "C" int palsgd_get_grad_norms(palsgd_ctx* ctx, double* sumsq, float* clip, void* stream)
+{
+    if (!ctx) return PALSGD_EINVAL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    DevState hs;
+    PALSGD_CUDA(ctx, cudaMemcpyAsync(&hs, ctx->tb.st, sizeof(hs), cudaMemcpyDeviceToHost, s));
+    PALSGD_CUDA(ctx, cudaStreamSynchronize(s));
+    for (uint32_t k = 0; k < ctx->cfg.K; ++k) {
+        if (sumsq) sumsq[k] = hs.sumsq[k];
+        if (clip) clip[k] = hs.clip[k];
+    }
     return PALSGD_OK;
 }
 

@@ -36,6 +36,11 @@ struct DevState {
     unsigned int       done;                 // CTAs that finished the current inner launch
     unsigned int       error;                // 0, or the code of a bounded wait that expired
     unsigned char      last_b[kMaxWorkers];  // decisions of the latest inner step
+    // global-norm gradient clipping (written by the norm kernel, read by the step kernels)
+    unsigned int       done_norm;            // CTAs that finished the current norm launch
+    unsigned int       pad_;
+    double             sumsq[kMaxWorkers];   // sum of squares of worker k's latest gradient
+    float              clip[kMaxWorkers];    // coefficient that gradient is scaled by (<= 1)
 };
 
 // Device pointer tables, indexed [k * n_seg + seg] (per-slot) or [seg].
@@ -55,6 +60,7 @@ struct Tables {
     float* const*       global;     // [n_seg]
     float* const*       outer_mom;  // [n_seg]
     DevState*           st;
+    double2*            norm_part;  // [n_chunks * K] per-work-item partial sums of squares (hi, lo)
 };
 
 struct InnerArgs {
@@ -67,6 +73,7 @@ struct InnerArgs {
     float    b1, b2, omb1, omb2, eps, decay;   // AdamW scalars, each rounded once from binary64
     float    mu, wd;       // momentum SGD scalars
     uint32_t chunk_major;  // 0: worker index fastest over work items; 1: chunk index fastest
+    uint32_t clip_on;      // 1: scale worker k's gradient by DevState::clip[k]
 };
 
 struct PullArgs {
@@ -93,6 +100,18 @@ struct DdpArgs {
     float    Kf;
     uint32_t sub_elems;    // elements per work item (a multiple of 4 * kThreads)
     uint32_t parts;        // work items per chunk
+    uint32_t clip_on;      // 1: scale the averaged gradient by DevState::clip[0]
+};
+
+// Gradient-norm pass of the global-norm clip.
+struct NormArgs {
+    Tables   tb;
+    uint64_t seed;
+    uint64_t thr;          // decision threshold: workers that pull this step are skipped
+    double   max_norm;     // clip threshold
+    float    Kf;
+    uint32_t ddp;          // 0: per-worker norms (Algorithm 1 phase); 1: norm of the averaged gradient
+    uint32_t group;        // consecutive chunks per work item (a function of the problem size only)
 };
 
 }  // namespace palsgd

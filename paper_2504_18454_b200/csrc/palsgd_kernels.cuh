@@ -15,12 +15,15 @@ namespace palsgd {
 
 // ---------------------------------------------------------------- element math
 
-struct AdamScalars { float b1, b2, omb1, omb2, bc1, bc2, decay, lr, eps; };
-struct SgdScalars  { float mu, wd, lr; };
+// clip: the global-norm clip coefficient the gradient is multiplied by first (1 = no clipping;
+// the multiplication by 1 is exact, so one code path serves both cases).
+struct AdamScalars { float b1, b2, omb1, omb2, bc1, bc2, decay, lr, eps; float clip = 1.f; };
+struct SgdScalars  { float mu, wd, lr; float clip = 1.f; };
 
 // AdamW with decoupled decay and bias correction (gradient branch, Eq. (1)).
 __device__ __forceinline__ void adamw_elem(float g, float& x, float& m, float& v, const AdamScalars& s)
 {
+    g = __fmul_rn(g, s.clip);
     m = __fadd_rn(__fmul_rn(s.b1, m), __fmul_rn(s.omb1, g));
     v = __fadd_rn(__fmul_rn(s.b2, v), __fmul_rn(s.omb2, __fmul_rn(g, g)));
     const float mh = __fdiv_rn(m, s.bc1);
@@ -32,6 +35,7 @@ __device__ __forceinline__ void adamw_elem(float g, float& x, float& m, float& v
 // Momentum SGD, L2 decay folded into the gradient (gradient branch, Eq. (1)).
 __device__ __forceinline__ void sgdm_elem(float g, float& x, float& buf, const SgdScalars& s)
 {
+    g = __fmul_rn(g, s.clip);
     const float gp = __fadd_rn(g, __fmul_rn(s.wd, x));
     buf = __fadd_rn(__fmul_rn(s.mu, buf), gp);
     x = __fsub_rn(x, __fmul_rn(s.lr, buf));
@@ -496,7 +500,7 @@ __global__ void __launch_bounds__(kThreads, MINB)
 palsgd_inner_kernel(const __grid_constant__ InnerArgs a)
 {
     __shared__ unsigned char s_pull[kMaxWorkers];
-    __shared__ float s_bc1[kMaxWorkers], s_bc2[kMaxWorkers];
+    __shared__ float s_bc1[kMaxWorkers], s_bc2[kMaxWorkers], s_clip[kMaxWorkers];
 
     const Tables& tb = a.tb;
     const uint32_t K = tb.K;
@@ -507,6 +511,7 @@ palsgd_inner_kernel(const __grid_constant__ InnerArgs a)
         const uint32_t k = threadIdx.x;
         const bool pull = draw_pull(a.seed, t, k, a.thr);
         s_pull[k] = pull;
+        s_clip[k] = a.clip_on ? st->clip[k] : 1.f;
         if (INNER == 0 && !pull) {                       // bias corrections for gradient step s_k + 1
             s_bc1[k] = (float)(1.0 - st->pow1[k] * a.beta1);
             s_bc2[k] = (float)(1.0 - st->pow2[k] * a.beta2);
@@ -521,8 +526,8 @@ palsgd_inner_kernel(const __grid_constant__ InnerArgs a)
         if (s_pull[k]) {
             pull_item<PREC, U, kThreads>(threadIdx.x, tb, k, ch, a.beta_pull);
         } else {
-            const AdamScalars as{a.b1, a.b2, a.omb1, a.omb2, s_bc1[k], s_bc2[k], a.decay, a.lr, a.eps};
-            const SgdScalars  ss{a.mu, a.wd, a.lr};
+            const AdamScalars as{a.b1, a.b2, a.omb1, a.omb2, s_bc1[k], s_bc2[k], a.decay, a.lr, a.eps, s_clip[k]};
+            const SgdScalars  ss{a.mu, a.wd, a.lr, s_clip[k]};
             grad_item<INNER, PREC, U, kThreads>(threadIdx.x, tb, k, ch, as, ss);
         }
     }
@@ -681,7 +686,8 @@ palsgd_ddp_kernel(const __grid_constant__ DdpArgs a)
         as.bc1 = (float)(1.0 - st->pow1[0] * a.beta1);
         as.bc2 = (float)(1.0 - st->pow2[0] * a.beta2);
     }
-    const SgdScalars ss{a.mu, a.wd, a.lr};
+    SgdScalars ss{a.mu, a.wd, a.lr};
+    if (a.clip_on) { as.clip = st->clip[0]; ss.clip = as.clip; }   // the clip applies to the averaged gradient
 
     const uint64_t n_items = (uint64_t)tb.n_chunks * a.parts;
     for (uint64_t item = blockIdx.x; item < n_items; item += gridDim.x) {

@@ -89,10 +89,37 @@ def _child(args) -> None:
         per = (16 if cfg.inner == 0 else 12) * (cfg.K + 1)      # both precisions: see include/palsgd.h
         return per * cfg.P / (e0.elapsed_time(e1) / reps) / 1e6
 
+    def time_norm(steps, ddp=False, warm=3):
+        # the norm pass alone = (clipped step) - (unclipped step), both timed over the same decisions
+        def loop(n):
+            ctx.set_counters(0, [0] * cfg.K, 0, stream)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            for i in range(warm + n):
+                if i == warm:
+                    e0.record()
+                ctx.ddp_step(cfg.lr, stream) if ddp else ctx.inner_step(cfg.lr, cfg.eta, stream)
+            e1.record()
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1)
+        ctx.set_grad_clip(0.0); base = loop(steps)
+        ctx.set_grad_clip(1.0); clipped = loop(steps)
+        ctx.set_grad_clip(0.0)
+        gsz = 2 if cfg.precision == 1 else 4
+        if ddp:
+            byts = steps * cfg.K * cfg.P * gsz
+        else:
+            byts = sum(0 if P.decision(cfg.decision_seed, warm + i, k, cfg.p) else gsz
+                       for i in range(steps) for k in range(cfg.K)) * cfg.P
+        return byts / (clipped - base) / 1e6, (clipped - base) / steps, base / steps
+
     for v in args.variants:
         ctx.set_tuning(P.TUNE_INNER_VARIANT, v)
         r = sorted(time_inner(args.steps) for _ in range(3))
         print(f"{cfg.name} chunk={chunk} inner variant={v}: {r[1]:.0f} GB/s (runs {r[0]:.0f}..{r[2]:.0f})", flush=True)
+    for ddp in (False, True):
+        r = sorted(time_norm(args.steps, ddp) for _ in range(3))[1]
+        print(f"{cfg.name} chunk={chunk} grad-norm pass ({'ddp' if ddp else 'per worker'}): {r[0]:.0f} GB/s of gradient "
+              f"bytes, {r[1]:.3f} ms on top of a {r[2]:.3f} ms step", flush=True)
     for sub in args.outer_subs:
         ctx.set_tuning(P.TUNE_OUTER_SUB_ELEMS, sub)
         r = sorted(time_outer() for _ in range(3))

@@ -136,6 +136,12 @@ class GpuRun:
     def ddp_step(self, lr):
         self.lib.ddp_step(lr, self.stream)
 
+    def set_grad_clip(self, max_norm):
+        self.lib.set_grad_clip(max_norm)
+
+    def grad_norms(self):
+        return self.lib.get_grad_norms(self.stream)
+
     def pseudo_sync(self, mask, beta):
         self.lib.pseudo_sync(mask, beta, self.stream)
 
