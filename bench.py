@@ -265,6 +265,8 @@ def run_ours(args, cfg):
 
     if args.inner_variant:
         ctx.set_tuning(P.TUNE_INNER_VARIANT, args.inner_variant)
+    if args.grad_clip > 0:
+        ctx.set_grad_clip(args.grad_clip)
     t_host = 0                                           # mirrors the library's step counter
     def one_step(ev_list=None):
         nonlocal t_host
@@ -418,6 +420,8 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(W.CONFIGS))
     ap.add_argument("--e2e-steps", type=int, default=0, help="0 = min(steps, H)")
     ap.add_argument("--inner-variant", type=int, default=0, help="palsgd_set_tuning(INNER_VARIANT); 0 = default")
+    ap.add_argument("--grad-clip", type=float, default=0.0,
+                    help="global-norm clip threshold (adds the norm pass to every step); 0 = off, the benchmark default")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-ddp", action="store_true", help="skip the separate timing of the DDP warm-up kernel")

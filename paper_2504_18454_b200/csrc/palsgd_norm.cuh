@@ -18,14 +18,16 @@ namespace palsgd {
 
 struct DD { double hi, lo; };
 
-// hi + lo += x, with hi + x split exactly into its rounded sum and the rounding error (Knuth's
-// TwoSum, six binary64 operations).  Measured on B200: ordering the operands with a comparison
-// and selects so that the three-operation form applies is slower, not faster.
+// hi + lo += x for x >= 0 and hi >= 0: hi + x is split exactly into its rounded sum and the
+// rounding error.  With the larger operand first the error is small - (s - big) (Dekker's
+// FastTwoSum): three binary64 operations and a comparison where the order-free form takes six.
 __device__ __forceinline__ void dd_accumulate(DD& a, double x)
 {
-    const double s  = __dadd_rn(a.hi, x);
-    const double bb = __dsub_rn(s, a.hi);
-    const double e  = __dadd_rn(__dsub_rn(a.hi, __dsub_rn(s, bb)), __dsub_rn(x, bb));
+    const bool   hi_big = a.hi >= x;
+    const double big    = hi_big ? a.hi : x;
+    const double small  = hi_big ? x : a.hi;
+    const double s = __dadd_rn(big, small);
+    const double e = __dsub_rn(small, __dsub_rn(s, big));
     a.hi = s;
     a.lo = __dadd_rn(a.lo, e);
 }
@@ -78,23 +80,46 @@ __device__ __forceinline__ DD dd_block_sum(DD v, DD* s_warp /* [kThreads / 32] *
 template <int PREC>
 __device__ __forceinline__ void sumsq_chunk(DD (&q)[4], const void* g, uint32_t len, bool vec)
 {
+    constexpr int U = 4;                                    // 128-bit loads in flight per thread
     uint32_t done = 0;
     if (vec) {
         if (PREC) {
             const uint4* g8 = static_cast<const uint4*>(g);
             const uint32_t n8 = len >> 3;
-            for (uint32_t i = threadIdx.x; i < n8; i += kThreads) {
-                float f[8]; unpack8(ld_stream(g8 + i), f);
+            for (uint32_t base = 0; base < n8; base += kThreads * U) {
+                uint4 R[U];
 #pragma unroll
-                for (int c = 0; c < 8; ++c) dd_square_in(q[c & 3], f[c]);
+                for (int u = 0; u < U; ++u) {
+                    const uint32_t i = base + u * kThreads + threadIdx.x;
+                    if (i < n8) R[u] = ld_stream(g8 + i);
+                }
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    const uint32_t i = base + u * kThreads + threadIdx.x;
+                    if (i < n8) {
+                        float f[8]; unpack8(R[u], f);
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) dd_square_in(q[c & 3], f[c]);
+                    }
+                }
             }
             done = n8 << 3;
         } else {
             const float4* g4 = static_cast<const float4*>(g);
             const uint32_t n4 = len >> 2;
-            for (uint32_t i = threadIdx.x; i < n4; i += kThreads) {
-                const float4 v = ld_stream(g4 + i);
-                dd_square_in(q[0], v.x); dd_square_in(q[1], v.y); dd_square_in(q[2], v.z); dd_square_in(q[3], v.w);
+            for (uint32_t base = 0; base < n4; base += kThreads * U) {
+                float4 R[U];
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    const uint32_t i = base + u * kThreads + threadIdx.x;
+                    if (i < n4) R[u] = ld_stream(g4 + i);
+                }
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    const uint32_t i = base + u * kThreads + threadIdx.x;
+                    if (i < n4) { dd_square_in(q[0], R[u].x); dd_square_in(q[1], R[u].y);
+                                  dd_square_in(q[2], R[u].z); dd_square_in(q[3], R[u].w); }
+                }
             }
             done = n4 << 2;
         }
