@@ -48,6 +48,9 @@ def lib() -> C.CDLL:
             f.restype = C.c_double
         L.palsgd_oracle_clip_coef.argtypes = [C.c_double, C.c_double]
         L.palsgd_oracle_clip_coef.restype = C.c_double
+        L.palsgd_oracle_schedule.argtypes = [C.c_int, C.c_uint64, C.c_uint64, C.c_uint64, C.c_double,
+                                             C.c_double, C.c_double]
+        L.palsgd_oracle_schedule.restype = C.c_double
         L.palsgd_oracle_set_threads.argtypes = [C.c_int]
         L.palsgd_oracle_set_threads.restype = None
         L.palsgd_oracle_get_threads.argtypes = []
@@ -101,6 +104,13 @@ def clip_coef(sumsq_: float, max_norm: float) -> float:
     return float(lib().palsgd_oracle_clip_coef(float(sumsq_), float(max_norm)))
 
 
+def schedule(kind: int, t: int, warmup: int, total: int, base: float, min_value: float = 0.0,
+             start_factor: float = 0.0) -> float:
+    """Linear warm-up, then constant (kind 0) or cosine annealing (kind 1)."""
+    return float(lib().palsgd_oracle_schedule(int(kind), int(t), int(warmup), int(total), float(base),
+                                              float(min_value), float(start_factor)))
+
+
 def set_threads(n: int) -> None:
     lib().palsgd_oracle_set_threads(int(n))
 
@@ -127,6 +137,9 @@ def _state_struct(real):
             ("last_b", C.POINTER(C.c_uint8)),
             ("max_grad_norm", C.c_double), ("forced_sumsq", C.POINTER(C.c_double)),
             ("sumsq", C.POINTER(C.c_double)), ("clipc", C.POINTER(C.c_double)),
+            ("outer_opt", C.c_int32), ("outer_beta1", C.c_double), ("outer_beta2", C.c_double),
+            ("outer_eps", C.c_double), ("outer_weight_decay", C.c_double), ("uv", ptr),
+            ("opow1", C.c_double), ("opow2", C.c_double),
         ]
 
     return State
@@ -148,7 +161,9 @@ class Oracle:
                  weight_decay: float = 0.01, momentum: float = 0.0,
                  outer_lr: float = 0.7, outer_momentum: float = 0.9,
                  outer_nesterov: bool = True, seed: int = 0, precision: int = 0,
-                 max_grad_norm: float = 0.0, dtype: str = "f32"):
+                 max_grad_norm: float = 0.0, outer_opt: int = 0, outer_beta1: float = 0.9,
+                 outer_beta2: float = 0.999, outer_eps: float = 1e-8, outer_weight_decay: float = 0.0,
+                 dtype: str = "f32"):
         x0 = np.asarray(x0)
         assert x0.ndim == 2 and x0.shape[0] == K, x0.shape
         self.dtype = dtype
@@ -159,6 +174,7 @@ class Oracle:
         self.v = np.zeros_like(self.x)
         self.xg = np.zeros(self.P, dtype=np_t)
         self.u = np.zeros(self.P, dtype=np_t)
+        self.uv = np.zeros(self.P, dtype=np_t) if outer_opt == 1 else None
         self.xw = np.zeros((self.K, self.P), dtype=np.uint16) if precision == 1 else None
         self.s = np.zeros(self.K, dtype=np.uint64)
         self.pow1 = np.ones(self.K, dtype=np.float64)
@@ -181,7 +197,10 @@ class Oracle:
             pow1=p_(self.pow1, C.c_double), pow2=p_(self.pow2, C.c_double),
             last_b=p_(self.last_b, C.c_uint8),
             max_grad_norm=float(max_grad_norm), forced_sumsq=None,
-            sumsq=p_(self.sumsq, C.c_double), clipc=p_(self.clipc, C.c_double))
+            sumsq=p_(self.sumsq, C.c_double), clipc=p_(self.clipc, C.c_double),
+            outer_opt=int(outer_opt), outer_beta1=outer_beta1, outer_beta2=outer_beta2,
+            outer_eps=outer_eps, outer_weight_decay=outer_weight_decay,
+            uv=p_(self.uv, ct) if self.uv is not None else None, opow1=1.0, opow2=1.0)
         L = lib()
         sfx = dtype
         self._init = getattr(L, f"palsgd_oracle_init_{sfx}")
@@ -209,6 +228,12 @@ class Oracle:
     @property
     def n_outer(self) -> int:
         return int(self._st.n_outer)
+
+    # schedules -----------------------------------------------------------
+    def set_outer_lr(self, lr: float) -> None:
+        """The outer learning rate may follow a schedule (warm-up, then cosine annealing): it is
+        an input of each synchronisation."""
+        self._st.outer_lr = float(lr)
 
     # gradient clipping ---------------------------------------------------
     def set_grad_clip(self, max_norm: float) -> None:

@@ -186,6 +186,28 @@ double palsgd_oracle_clip_coef(double sumsq, double max_norm)
     return c < 1.0 ? c : 1.0;
 }
 
+/* ---- learning-rate schedules ----------------------------------------------- */
+
+/* Value at step t of a schedule with a linear warm-up followed by a constant
+ * (kind 0) or by cosine annealing (kind 1), the form the paper's experiments use
+ * for the outer learning rate ("a warm-up period ... followed by cosine
+ * annealing", Appendix B):
+ *   t <  warmup : base * (start_factor + (1 - start_factor) * t / warmup)
+ *   t >= warmup : kind 0: base
+ *                 kind 1: min + (base - min) * (1 + cos(pi * tau / (total - warmup))) / 2,
+ *                         tau = min(t, total) - warmup           (stays at min after total) */
+double palsgd_oracle_schedule(int kind, uint64_t t, uint64_t warmup, uint64_t total,
+                              double base, double min_value, double start_factor)
+{
+    const double pi = 3.14159265358979323846;
+    if (t < warmup)
+        return base * (start_factor + (1.0 - start_factor) * (double)t / (double)warmup);
+    if (kind == 0 || total <= warmup) return base;
+    uint64_t tt = t < total ? t : total;
+    double tau = (double)(tt - warmup);
+    return min_value + (base - min_value) * (1.0 + cos(pi * tau / (double)(total - warmup))) / 2.0;
+}
+
 /* ---- thread count of the element loops (timing harness only) -------------- */
 #ifdef _OPENMP
 void palsgd_oracle_set_threads(int n) { if (n > 0) omp_set_num_threads(n); }

@@ -77,6 +77,12 @@ typedef struct {
                                 computing them (sampled replays of a large run)   */
     double   *sumsq;         /* [K] sum of squares of the latest gradients seen    */
     double   *clipc;         /* [K] coefficient the latest gradient was scaled by  */
+    /* OuterOPT variants of the optimizer ablation (Appendix D): 0 = SGD with
+     * (Nesterov) momentum as above, 1 = AdamW applied to the outer gradient    */
+    int32_t   outer_opt;
+    double    outer_beta1, outer_beta2, outer_eps, outer_weight_decay;
+    REAL     *uv;            /* [P] second outer moment (outer_opt = 1) or NULL    */
+    double    opow1, opow2;  /* outer_beta1^n_outer, outer_beta2^n_outer           */
 } FN(state);
 
 static uint16_t to_bf16(REAL a)
@@ -119,6 +125,11 @@ void FN(init)(FN(state) *st)
         refresh_working(st, k);
     }
     st->t = 0; st->n_outer = 0;
+    st->opow1 = 1.0; st->opow2 = 1.0;
+    if (st->uv) {
+        #pragma omp parallel for schedule(static)
+        for (int64_t i = 0; i < (int64_t)P; ++i) st->uv[i] = (REAL)0;
+    }
 }
 
 /* Eq. (2): x_k <- x_k - beta (x_k - x), beta = alpha_t eta_t / p.
@@ -251,12 +262,35 @@ void FN(outer_sync)(FN(state) *st)
     const uint32_t K = st->K;
     const size_t P = st->P;
     const REAL mu = (REAL)st->outer_momentum, lr = (REAL)st->outer_lr;
+    /* OuterOPT = AdamW on the outer gradient Delta (one of the ablation's choices): the textbook
+     * form used for InnerOPT, with u as first and uv as second moment and n_outer + 1 as step count */
+    if (st->outer_opt == 1) {
+        st->opow1 *= st->outer_beta1;
+        st->opow2 *= st->outer_beta2;
+    }
+    const REAL ob1 = (REAL)st->outer_beta1, ob2 = (REAL)st->outer_beta2;
+    const REAL oomb1 = (REAL)(1.0 - st->outer_beta1), oomb2 = (REAL)(1.0 - st->outer_beta2);
+    const REAL obc1 = (REAL)(1.0 - st->opow1), obc2 = (REAL)(1.0 - st->opow2);
+    const REAL odecay = (REAL)(1.0 - st->outer_lr * st->outer_weight_decay);
+    const REAL oeps = (REAL)st->outer_eps;
     #pragma omp parallel for schedule(static)
     for (int64_t i = 0; i < (int64_t)P; ++i) {
         REAL sum = st->x[i];
         for (uint32_t k = 1; k < K; ++k) sum = sum + st->x[(size_t)k * P + i];
         REAL xbar  = sum / (REAL)K;
         REAL delta = st->xg[i] - xbar;
+        if (st->outer_opt == 1) {
+            REAL mi = ob1 * st->u[i] + oomb1 * delta;
+            REAL vi = ob2 * st->uv[i] + oomb2 * (delta * delta);
+            REAL mhat = mi / obc1;
+            REAL vhat = vi / obc2;
+            REAL xi = st->xg[i] * odecay;
+            REAL root = sizeof(REAL) == 4 ? (REAL)sqrtf((float)vhat) : (REAL)sqrt((double)vhat);
+            xi = xi - lr * (mhat / (root + oeps));
+            st->u[i] = mi; st->uv[i] = vi; st->xg[i] = xi;
+            for (uint32_t k = 0; k < K; ++k) st->x[(size_t)k * P + i] = xi;
+            continue;
+        }
         REAL ui    = mu * st->u[i] + delta;
         REAL step  = st->outer_nesterov ? (delta + mu * ui) : ui;
         REAL xnew  = st->xg[i] - lr * step;
