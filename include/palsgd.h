@@ -62,6 +62,8 @@ typedef enum palsgd_status {
 
 enum { PALSGD_INNER_ADAMW = 0, PALSGD_INNER_SGDM = 1 };
 enum { PALSGD_PREC_FP32 = 0, PALSGD_PREC_BF16_MASTER = 1 };
+enum { PALSGD_OUTER_SGD = 0, PALSGD_OUTER_ADAMW = 1 };
+enum { PALSGD_SCHED_WARMUP_CONSTANT = 0, PALSGD_SCHED_WARMUP_COSINE = 1 };
 
 /* Algorithm 1's data line: K, p, H, InnerOPT, OuterOPT.  (alpha_t and eta_t are
  * per-call arguments because the paper indexes them by t.) */
@@ -79,6 +81,12 @@ typedef struct palsgd_config {
     int32_t  outer_nesterov;  /*   (1, 0, 0) is plain averaging (Local SGD / Theorem 1)          */
     int32_t  precision;       /* PALSGD_PREC_FP32 | PALSGD_PREC_BF16_MASTER                      */
     uint64_t seed;            /* seed of the decision stream                                     */
+    /* OuterOPT variants of the optimizer ablation (Appendix D).  PALSGD_OUTER_SGD uses
+     * outer_lr / outer_momentum / outer_nesterov above; PALSGD_OUTER_ADAMW applies AdamW to
+     * the outer gradient with the four constants below and needs palsgd_buffers.outer_v.     */
+    int32_t  outer_opt;       /* PALSGD_OUTER_SGD | PALSGD_OUTER_ADAMW                           */
+    int32_t  reserved_;       /* set to 0                                                        */
+    double   outer_beta1, outer_beta2, outer_eps, outer_weight_decay;
 } palsgd_config;
 
 /* Caller-owned device buffers.  Arrays of K*n_tensors pointers are indexed
@@ -92,7 +100,10 @@ typedef struct palsgd_buffers {
     float* const*      m;          /* [K*n] AdamW first moment / SGD momentum buffer             */
     float* const*      v;          /* [K*n] AdamW second moment; NULL for SGD                    */
     float* const*      global;     /* [n]   global model copy x (written by init)                */
-    float* const*      outer_mom;  /* [n]   OuterOPT momentum buffer u (zeroed by init)          */
+    float* const*      outer_mom;  /* [n]   OuterOPT momentum buffer u (zeroed by init); first
+                                      moment of the outer gradient for PALSGD_OUTER_ADAMW         */
+    float* const*      outer_v;    /* [n]   second moment for PALSGD_OUTER_ADAMW (zeroed by init),
+                                      else NULL                                                  */
 } palsgd_buffers;
 
 /*
@@ -161,11 +172,35 @@ int palsgd_pseudo_sync(palsgd_ctx* ctx, uint64_t worker_mask, double beta, void*
  *   u = mu*u + Delta;  x_g = x_g - lr_out*(Delta + mu*u)   (Nesterov; Eq. (4))
  *                      x_g = x_g - lr_out*u                (outer_nesterov = 0)
  *   x_k = x_g for every k  (Sec. 3.1: every worker restarts from the global model)
+ * With PALSGD_OUTER_ADAMW (the ablation's AdamW OuterOPT) the update of x_g is instead, with
+ * n = n_outer + 1 and the outer_* constants of the configuration:
+ *   u = ob1*u + (1-ob1)*Delta;  v = ob2*v + (1-ob2)*(Delta*Delta);
+ *   uh = u / (1-ob1^n);  vh = v / (1-ob2^n);
+ *   x_g = x_g * fl32(1 - lr_out*owd);  x_g = x_g - lr_out * (uh / (sqrt(vh) + oeps))
+ * lr_out is the configuration's outer_lr or the latest palsgd_set_outer_lr value.
  * Inner optimizer state is kept.  n_outer += 1.  BF16_MASTER: masters are
  * averaged; masters and bf16 working copies are rewritten.
  * Errors: EINVAL (NULL ctx); ECUDA.
  */
 int palsgd_outer_sync(palsgd_ctx* ctx, void* stream);
+
+/* The outer learning rate of the following outer syncs (it may follow a schedule, e.g. the
+ * warm-up + cosine annealing of Appendix B: see palsgd_schedule_value).  Errors: EINVAL. */
+int palsgd_set_outer_lr(palsgd_ctx* ctx, double outer_lr);
+
+/*
+ * Pure host function: the value at step t of a schedule with a linear warm-up over
+ * `warmup` steps from base*start_factor to base, followed by a constant
+ * (PALSGD_SCHED_WARMUP_CONSTANT) or by cosine annealing down to min_value at step `total`
+ * (PALSGD_SCHED_WARMUP_COSINE; Appendix B: "a warm-up period ... followed by cosine annealing"):
+ *   t <  warmup: base * (start_factor + (1 - start_factor) * t / warmup)
+ *   t >= warmup: base, or min_value + (base - min_value) * (1 + cos(pi*tau/(total - warmup))) / 2
+ *                with tau = min(t, total) - warmup.
+ * Returns NaN for an unknown kind or non-finite arguments.  Feed the result to
+ * palsgd_inner_step / palsgd_step (alpha_t, eta_t) or palsgd_set_outer_lr.
+ */
+double palsgd_schedule_value(int kind, uint64_t t, uint64_t warmup, uint64_t total, double base,
+                             double min_value, double start_factor);
 
 /* Algorithm 1, one iteration t: palsgd_inner_step, then palsgd_outer_sync when
  * the number of completed steps is a multiple of H. */

@@ -9,6 +9,11 @@ from .binding import (  # noqa: F401
     Palsgd,
     PalsgdError,
     decision,
+    schedule_value,
+    OUTER_SGD,
+    OUTER_ADAMW,
+    SCHED_WARMUP_CONSTANT,
+    SCHED_WARMUP_COSINE,
     outer_sync_noalloc,
     NOALLOC_SCRATCH_BYTES,
     lib,

@@ -17,7 +17,7 @@ from .binding import INNER_ADAMW, PREC_BF16_MASTER, Palsgd
 
 class ReplicaArena:
     def __init__(self, numel: Sequence[int], K: int, *, precision: int, inner: int,
-                 device: torch.device | str = "cuda"):
+                 device: torch.device | str = "cuda", outer_adamw: bool = False):
         self.numel = [int(n) for n in numel]
         self.K, self.P = int(K), int(sum(self.numel))
         self.precision, self.inner = precision, inner
@@ -33,6 +33,8 @@ class ReplicaArena:
             self.t["v"] = mk(K, torch.float32)
         if bf:
             self.t["master"] = mk(K, torch.float32)
+        if outer_adamw:                          # second moment of AdamW as OuterOPT
+            self.t["outer_v"] = mk(1, torch.float32)
         starts = [0]
         for n in self.numel:
             starts.append(starts[-1] + n)
@@ -59,5 +61,5 @@ class ReplicaArena:
         v = {k: self.views(k) for k in self.t}
         return Palsgd(K=self.K, numel=self.numel, params=v["param"], grads=v["grad"], m=v["m"],
                       v=v.get("v"), master=v.get("master"), global_=v["global_"][0],
-                      outer_mom=v["outer_mom"][0], precision=self.precision, inner=self.inner,
-                      stream=stream, **cfg)
+                      outer_mom=v["outer_mom"][0], outer_v=v["outer_v"][0] if "outer_v" in v else None,
+                      precision=self.precision, inner=self.inner, stream=stream, **cfg)

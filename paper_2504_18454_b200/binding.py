@@ -10,6 +10,8 @@ LIB_PATH = HERE / "libpalsgd.so"
 
 INNER_ADAMW, INNER_SGDM = 0, 1
 PREC_FP32, PREC_BF16_MASTER = 0, 1
+OUTER_SGD, OUTER_ADAMW = 0, 1
+SCHED_WARMUP_CONSTANT, SCHED_WARMUP_COSINE = 0, 1
 TUNE_INNER_GRID_CAP, TUNE_OUTER_GRID_CAP, TUNE_INNER_VARIANT, TUNE_PIPE_STAGES = 0, 1, 2, 3
 TUNE_CHUNK_MAJOR, TUNE_OUTER_SUB_ELEMS, TUNE_DDP_SUB_ELEMS = 4, 5, 6
 MAX_WORKERS = 64
@@ -28,12 +30,15 @@ class Config(C.Structure):
         ("weight_decay", C.c_double), ("momentum", C.c_double),
         ("outer_lr", C.c_double), ("outer_momentum", C.c_double),
         ("outer_nesterov", C.c_int32), ("precision", C.c_int32), ("seed", C.c_uint64),
+        ("outer_opt", C.c_int32), ("reserved_", C.c_int32),
+        ("outer_beta1", C.c_double), ("outer_beta2", C.c_double), ("outer_eps", C.c_double),
+        ("outer_weight_decay", C.c_double),
     ]
 
 
 class Buffers(C.Structure):
     _fields_ = [(n, C.POINTER(C.c_void_p)) for n in
-                ("param", "grad", "master", "m", "v", "global_", "outer_mom")]
+                ("param", "grad", "master", "m", "v", "global_", "outer_mom", "outer_v")]
 
 
 _lib: Optional[C.CDLL] = None
@@ -55,6 +60,11 @@ def lib() -> C.CDLL:
     L.palsgd_pseudo_sync.argtypes = [vp, C.c_uint64, C.c_double, vp]
     L.palsgd_ddp_step.argtypes = [vp, C.c_double, vp]
     L.palsgd_ddp_step.restype = C.c_int
+    L.palsgd_set_outer_lr.argtypes = [vp, C.c_double]
+    L.palsgd_set_outer_lr.restype = C.c_int
+    L.palsgd_schedule_value.argtypes = [C.c_int, C.c_uint64, C.c_uint64, C.c_uint64, C.c_double, C.c_double,
+                                        C.c_double]
+    L.palsgd_schedule_value.restype = C.c_double
     L.palsgd_set_grad_clip.argtypes = [vp, C.c_double]
     L.palsgd_set_grad_clip.restype = C.c_int
     L.palsgd_get_grad_norms.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_float), vp]
@@ -95,6 +105,13 @@ def decision(seed: int, t: int, k: int, p: float) -> int:
     if rc < 0:
         raise PalsgdError(rc, "palsgd_decision")
     return rc
+
+
+def schedule_value(kind: int, t: int, warmup: int, total: int, base: float, min_value: float = 0.0,
+                   start_factor: float = 0.0) -> float:
+    """palsgd_schedule_value: linear warm-up, then constant or cosine annealing (pure host function)."""
+    return float(lib().palsgd_schedule_value(int(kind), int(t), int(warmup), int(total), float(base),
+                                             float(min_value), float(start_factor)))
 
 
 def _ptr_array(ptrs: Sequence[int]):
@@ -142,15 +159,19 @@ class Palsgd:
                  inner: int = INNER_ADAMW, beta1: float = 0.9, beta2: float = 0.999,
                  eps: float = 1e-8, weight_decay: float = 0.01, momentum: float = 0.0,
                  outer_lr: float = 0.7, outer_momentum: float = 0.9, outer_nesterov: bool = True,
-                 precision: int = PREC_FP32, seed: int = 0, stream: int = 0):
+                 precision: int = PREC_FP32, seed: int = 0, stream: int = 0,
+                 outer_opt: int = OUTER_SGD, outer_v=None, outer_beta1: float = 0.9, outer_beta2: float = 0.999,
+                 outer_eps: float = 1e-8, outer_weight_decay: float = 0.0):
         self._ctx = C.c_void_p()
         self.K, self.H, self.n = int(K), int(H), len(numel)
         self.numel = [int(x) for x in numel]
-        self._keep = (params, grads, m, v, master, global_, outer_mom)
+        self._keep = (params, grads, m, v, master, global_, outer_mom, outer_v)
         cfg = Config(K=K, inner=inner, H=H, p=p, beta1=beta1, beta2=beta2, eps=eps,
                      weight_decay=weight_decay, momentum=momentum, outer_lr=outer_lr,
                      outer_momentum=outer_momentum, outer_nesterov=int(bool(outer_nesterov)),
-                     precision=precision, seed=seed)
+                     precision=precision, seed=seed, outer_opt=outer_opt, reserved_=0,
+                     outer_beta1=outer_beta1, outer_beta2=outer_beta2, outer_eps=outer_eps,
+                     outer_weight_decay=outer_weight_decay)
         arrs = {
             "param": _ptr_array(_data_ptrs(params)),
             "grad": _ptr_array(_data_ptrs(grads)),
@@ -159,6 +180,7 @@ class Palsgd:
             "v": _ptr_array(_data_ptrs(v)) if v is not None else None,
             "global_": _ptr_array([int(t.data_ptr()) for t in global_]),
             "outer_mom": _ptr_array([int(t.data_ptr()) for t in outer_mom]),
+            "outer_v": _ptr_array([int(t.data_ptr()) for t in outer_v]) if outer_v is not None else None,
         }
         bufs = Buffers(**{k: (C.cast(a, C.POINTER(C.c_void_p)) if a is not None else None)
                           for k, a in arrs.items()})
@@ -219,6 +241,9 @@ class Palsgd:
     def set_counters(self, t: int, s: Sequence[int], n_outer: int, stream: int = 0) -> None:
         arr = (C.c_uint64 * self.K)(*[int(x) for x in s])
         self._check(lib().palsgd_set_counters(self._ctx, t, arr, n_outer, C.c_void_p(stream)), "palsgd_set_counters")
+
+    def set_outer_lr(self, outer_lr: float) -> None:
+        self._check(lib().palsgd_set_outer_lr(self._ctx, outer_lr), "palsgd_set_outer_lr")
 
     def set_grad_clip(self, max_norm: float) -> None:
         self._check(lib().palsgd_set_grad_clip(self._ctx, max_norm), "palsgd_set_grad_clip")

@@ -51,6 +51,8 @@ struct palsgd_ctx {
     uint32_t outer_sub_elems = kOuterSubElems;    // elements per work item of the outer kernel
     uint32_t ddp_sub_elems = kDdpSubElems;        // elements per work item of the DDP warm-up kernel
     double max_grad_norm = 0.0;                   // global-norm clip threshold, 0 = off
+    double outer_lr = 0.0;                        // OuterOPT learning rate of the next sync
+    double opow1 = 1.0, opow2 = 1.0;              // outer_beta^n_outer (AdamW as OuterOPT), running products
     int sm_count = 0, smem_optin = 0;             // device attributes read at init
     std::string cuda_err;
 };
@@ -93,6 +95,12 @@ int validate_config(const palsgd_config* c)
     }
     if (!finite_nonneg(c->weight_decay)) return PALSGD_EINVAL;
     if (!std::isfinite(c->outer_lr) || !finite_nonneg(c->outer_momentum)) return PALSGD_EINVAL;
+    if (c->outer_opt != PALSGD_OUTER_SGD && c->outer_opt != PALSGD_OUTER_ADAMW) return PALSGD_EINVAL;
+    if (c->outer_opt == PALSGD_OUTER_ADAMW) {
+        if (!(c->outer_beta1 >= 0.0 && c->outer_beta1 < 1.0) || !(c->outer_beta2 >= 0.0 && c->outer_beta2 < 1.0))
+            return PALSGD_EINVAL;
+        if (!finite_nonneg(c->outer_eps) || !finite_nonneg(c->outer_weight_decay)) return PALSGD_EINVAL;
+    }
     return PALSGD_OK;
 }
 
@@ -131,9 +139,20 @@ OuterArgs outer_args(const palsgd_ctx* ctx)
     OuterArgs a{};
     a.tb = ctx->tb;
     a.mu = (float)ctx->cfg.outer_momentum;
-    a.lr = (float)ctx->cfg.outer_lr;
+    a.lr = (float)ctx->outer_lr;
     a.Kf = (float)ctx->cfg.K;
     a.nesterov = ctx->cfg.outer_nesterov;
+    if (ctx->cfg.outer_opt == PALSGD_OUTER_ADAMW) {          // scalars of outer step n_outer + 1
+        const palsgd_config& c = ctx->cfg;
+        a.ob1 = (float)c.outer_beta1;
+        a.ob2 = (float)c.outer_beta2;
+        a.oomb1 = (float)(1.0 - c.outer_beta1);
+        a.oomb2 = (float)(1.0 - c.outer_beta2);
+        a.obc1 = (float)(1.0 - ctx->opow1 * c.outer_beta1);
+        a.obc2 = (float)(1.0 - ctx->opow2 * c.outer_beta2);
+        a.odecay = (float)(1.0 - ctx->outer_lr * c.outer_weight_decay);
+        a.oeps = (float)c.outer_eps;
+    }
     a.sub_elems = ctx->outer_sub_elems;
     a.parts = (ctx->chunk_elems + a.sub_elems - 1) / a.sub_elems;
     return a;
@@ -275,6 +294,8 @@ extern "C" int palsgd_init(palsgd_ctx** out, const palsgd_config* cfg, size_t n_
     if (!bufs->param || !bufs->grad || !bufs->m || !bufs->global || !bufs->outer_mom) return PALSGD_EINVAL;
     if (bf && !bufs->master) return PALSGD_EINVAL;
     if (adam && !bufs->v) return PALSGD_EINVAL;
+    const bool oadam = cfg->outer_opt == PALSGD_OUTER_ADAMW;
+    if (oadam && !bufs->outer_v) return PALSGD_EINVAL;
 
     // which buffer kinds exist, and their element sizes
     const size_t ps = elem_size_param(cfg->precision);
@@ -296,6 +317,10 @@ extern "C" int palsgd_init(palsgd_ctx** out, const palsgd_config* cfg, size_t n_
         }
         if ((!bufs->global[j] || !bufs->outer_mom[j]) && numel[j] > 0) return PALSGD_EINVAL;
         if (!aligned(bufs->global[j], 4) || !aligned(bufs->outer_mom[j], 4)) return PALSGD_EALIGN;
+        if (oadam) {
+            if (!bufs->outer_v[j] && numel[j] > 0) return PALSGD_EINVAL;
+            if (!aligned(bufs->outer_v[j], 4)) return PALSGD_EALIGN;
+        }
     }
 
     palsgd_ctx* ctx = new (std::nothrow) palsgd_ctx();
@@ -305,6 +330,7 @@ extern "C" int palsgd_init(palsgd_ctx** out, const palsgd_config* cfg, size_t n_
     ctx->numel.assign(numel, numel + n_tensors);
     ctx->P = P;
     ctx->thr = threshold_of(cfg->p);
+    ctx->outer_lr = cfg->outer_lr;
     ctx->h_grad_dev.assign(bufs->grad, bufs->grad + (size_t)K * n_tensors);
     ctx->h_global_dev.assign(bufs->global, bufs->global + n_tensors);
 
@@ -321,6 +347,8 @@ extern "C" int palsgd_init(palsgd_ctx** out, const palsgd_config* cfg, size_t n_
         }
         const char* ga = reinterpret_cast<const char*>(bufs->global[j]);
         const char* ua = reinterpret_cast<const char*>(bufs->outer_mom[j]);
+        if (oadam && reinterpret_cast<const char*>(bufs->outer_v[j]) + numel[j] * 4 !=
+                         reinterpret_cast<const char*>(bufs->outer_v[j + 1])) return false;
         return ga + numel[j] * 4 == reinterpret_cast<const char*>(bufs->global[j + 1]) &&
                ua + numel[j] * 4 == reinterpret_cast<const char*>(bufs->outer_mom[j + 1]);
     };
@@ -346,7 +374,8 @@ extern "C" int palsgd_init(palsgd_ctx** out, const palsgd_config* cfg, size_t n_
     std::vector<Chunk> chunks;
     for (size_t s = 0; s < n_seg; ++s) {
         const Segment& sg = ctx->segs[s];
-        bool vec = aligned(bufs->global[sg.first_tensor], 16) && aligned(bufs->outer_mom[sg.first_tensor], 16);
+        bool vec = aligned(bufs->global[sg.first_tensor], 16) && aligned(bufs->outer_mom[sg.first_tensor], 16) &&
+                   (!oadam || aligned(bufs->outer_v[sg.first_tensor], 16));
         for (uint32_t k = 0; k < K && vec; ++k)
             for (const Kind& kd : kinds)
                 if (kd.present && !aligned(buf_ptr(bufs, kd.id, (size_t)k * n_tensors + sg.first_tensor), 16))
@@ -368,7 +397,7 @@ extern "C" int palsgd_init(palsgd_ctx** out, const palsgd_config* cfg, size_t n_
     size_t off_state = 0;
     size_t off_chunks = round_up(sizeof(DevState), 256);
     size_t off_tabs = round_up(off_chunks + chunks.size() * sizeof(Chunk), 256);
-    const size_t off_norm = off_tabs + 5 * round_up(per_slot, 256) + 2 * round_up(per_seg, 256) + 256;
+    const size_t off_norm = off_tabs + 5 * round_up(per_slot, 256) + 3 * round_up(per_seg, 256) + 256;
     const size_t total = off_norm + round_up(chunks.size() * K * sizeof(double2), 256) + 256;
     std::vector<char> host(total, 0);
     DevState hs{};
@@ -425,6 +454,7 @@ extern "C" int palsgd_init(palsgd_ctx** out, const palsgd_config* cfg, size_t n_
     tb.v = adam ? static_cast<float* const*>(fill_slot_table(4)) : nullptr;
     tb.global = static_cast<float* const*>(fill_seg_table(bufs->global));
     tb.outer_mom = static_cast<float* const*>(fill_seg_table(bufs->outer_mom));
+    tb.outer_v = oadam ? static_cast<float* const*>(fill_seg_table(bufs->outer_v)) : nullptr;
     tb.xf = static_cast<float* const*>(bf ? t_master : t_param);
     tb.xw = bf ? static_cast<__nv_bfloat16* const*>(t_param) : nullptr;
     tb.norm_part = reinterpret_cast<double2*>(d + off_norm);
@@ -549,11 +579,18 @@ extern "C" int palsgd_outer_sync(palsgd_ctx* ctx, void* stream)
         const unsigned grid = grid_for((uint64_t)ctx->tb.n_chunks * a.parts, ctx->grid_cap_outer);
         cudaStream_t s = static_cast<cudaStream_t>(stream);
         const bool bf = ctx->cfg.precision == PALSGD_PREC_BF16_MASTER;
+        const bool oadam = ctx->cfg.outer_opt == PALSGD_OUTER_ADAMW;
         int rc = launch_checked(ctx, [&] {
-            if (bf) palsgd_outer_kernel<1><<<grid, kThreads, 0, s>>>(a);
-            else    palsgd_outer_kernel<0><<<grid, kThreads, 0, s>>>(a);
+            if (bf && oadam)       palsgd_outer_kernel<1, 1><<<grid, kThreads, 0, s>>>(a);
+            else if (bf)           palsgd_outer_kernel<1, 0><<<grid, kThreads, 0, s>>>(a);
+            else if (oadam)        palsgd_outer_kernel<0, 1><<<grid, kThreads, 0, s>>>(a);
+            else                   palsgd_outer_kernel<0, 0><<<grid, kThreads, 0, s>>>(a);
         });
         if (rc) return rc;
+    }
+    if (ctx->cfg.outer_opt == PALSGD_OUTER_ADAMW) {
+        ctx->opow1 *= ctx->cfg.outer_beta1;
+        ctx->opow2 *= ctx->cfg.outer_beta2;
     }
     ctx->n_outer += 1;
     return PALSGD_OK;
@@ -670,7 +707,34 @@ extern "C" int palsgd_set_counters(palsgd_ctx* ctx, uint64_t t, const uint64_t* 
     PALSGD_CUDA(ctx, cudaStreamSynchronize(s));          // hs lives on this stack frame
     ctx->t = t;
     ctx->n_outer = n_outer;
+    ctx->opow1 = ctx->opow2 = 1.0;
+    if (ctx->cfg.outer_opt == PALSGD_OUTER_ADAMW)
+        for (uint64_t i = 0; i < n_outer; ++i) {             // the running products of n_outer syncs
+            ctx->opow1 *= ctx->cfg.outer_beta1;
+            ctx->opow2 *= ctx->cfg.outer_beta2;
+            if (ctx->opow1 == 0.0 && ctx->opow2 == 0.0) break;
+        }
     return PALSGD_OK;
+}
+
+extern "C" int palsgd_set_outer_lr(palsgd_ctx* ctx, double outer_lr)
+{
+    if (!ctx || !std::isfinite(outer_lr)) return PALSGD_EINVAL;
+    ctx->outer_lr = outer_lr;
+    return PALSGD_OK;
+}
+
+extern "C" double palsgd_schedule_value(int kind, uint64_t t, uint64_t warmup, uint64_t total, double base,
+                                        double min_value, double start_factor)
+{
+    if ((kind != PALSGD_SCHED_WARMUP_CONSTANT && kind != PALSGD_SCHED_WARMUP_COSINE) || !std::isfinite(base) ||
+        !std::isfinite(min_value) || !std::isfinite(start_factor))
+        return std::nan("");
+    if (t < warmup) return base * (start_factor + (1.0 - start_factor) * (double)t / (double)warmup);
+    if (kind == PALSGD_SCHED_WARMUP_CONSTANT || total <= warmup) return base;
+    const double kPi = 3.14159265358979323846;
+    const double tau = (double)((t < total ? t : total) - warmup);
+    return min_value + (base - min_value) * (1.0 + std::cos(kPi * tau / (double)(total - warmup))) / 2.0;
 }
 
 extern "C" int palsgd_set_grad_clip(palsgd_ctx* ctx, double max_norm)

@@ -59,6 +59,7 @@ struct Tables {
     float* const*       v;          // nullptr table entries for SGD
     float* const*       global;     // [n_seg]
     float* const*       outer_mom;  // [n_seg]
+    float* const*       outer_v;    // [n_seg] second outer moment (AdamW as OuterOPT) or nullptr
     DevState*           st;
     double2*            norm_part;  // [n_chunks * K] per-work-item partial sums of squares (hi, lo)
 };
@@ -86,6 +87,7 @@ struct OuterArgs {
     Tables tb;
     float  mu, lr, Kf;
     int    nesterov;
+    float  ob1, ob2, oomb1, oomb2, obc1, obc2, odecay, oeps;   // AdamW as OuterOPT (step n_outer + 1)
     uint32_t sub_elems;    // elements per work item (a multiple of 4 * kThreads)
     uint32_t parts;        // work items per chunk = ceil(chunk_elems / sub_elems)
 };

@@ -581,10 +581,22 @@ __device__ __forceinline__ float outer_elem(float sum, float Kf, float xg, float
     return __fsub_rn(xg, __fmul_rn(lr, step));
 }
 
-template <int PREC>
+// OuterOPT = AdamW on the outer gradient: the inner optimizer's element formula with
+// g = Delta, x = x_g, first moment u and second moment uv.
+__device__ __forceinline__ float outer_elem_adamw(float sum, float Kf, float xg, float& u, float& uv, const AdamScalars& s)
+{
+    const float xbar  = __fdiv_rn(sum, Kf);
+    const float delta = __fsub_rn(xg, xbar);
+    adamw_elem(delta, xg, u, uv, s);
+    return xg;
+}
+
+// OOPT: 0 = SGD with (Nesterov) momentum, 1 = AdamW (one more state stream).
+template <int PREC, int OOPT>
 __global__ void __launch_bounds__(kThreads)
 palsgd_outer_kernel(const __grid_constant__ OuterArgs a)
 {
+    const AdamScalars os{a.ob1, a.ob2, a.oomb1, a.oomb2, a.obc1, a.obc2, a.odecay, a.lr, a.oeps};
     __shared__ float* s_x[kMaxWorkers];
     __shared__ __nv_bfloat16* s_w[kMaxWorkers];
     const Tables& tb = a.tb;
@@ -608,6 +620,7 @@ palsgd_outer_kernel(const __grid_constant__ OuterArgs a)
         __syncthreads();
         float* xg = tb.global[seg] + ch.off;
         float* um = tb.outer_mom[seg] + ch.off;
+        float* uv = OOPT ? tb.outer_v[seg] + ch.off : nullptr;
 
         uint32_t done = 0;
         if (ch.seg & kSegVecFlag) {
@@ -615,6 +628,8 @@ palsgd_outer_kernel(const __grid_constant__ OuterArgs a)
             for (uint32_t i = threadIdx.x; i < n4; i += kThreads) {
                 const float4 Q = __ldcs(reinterpret_cast<const float4*>(xg) + i);
                 float4 Um = __ldcs(reinterpret_cast<const float4*>(um) + i);
+                float4 Uv = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (OOPT) Uv = __ldcs(reinterpret_cast<const float4*>(uv) + i);
                 float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
                 for (uint32_t k0 = 0; k0 < K; k0 += B) {
                     float4 R[B];
@@ -630,10 +645,18 @@ palsgd_outer_kernel(const __grid_constant__ OuterArgs a)
                         }
                 }
                 float4 N;
-                N.x = outer_elem(acc.x, a.Kf, Q.x, Um.x, a.mu, a.lr, a.nesterov);
-                N.y = outer_elem(acc.y, a.Kf, Q.y, Um.y, a.mu, a.lr, a.nesterov);
-                N.z = outer_elem(acc.z, a.Kf, Q.z, Um.z, a.mu, a.lr, a.nesterov);
-                N.w = outer_elem(acc.w, a.Kf, Q.w, Um.w, a.mu, a.lr, a.nesterov);
+                if (OOPT) {
+                    N.x = outer_elem_adamw(acc.x, a.Kf, Q.x, Um.x, Uv.x, os);
+                    N.y = outer_elem_adamw(acc.y, a.Kf, Q.y, Um.y, Uv.y, os);
+                    N.z = outer_elem_adamw(acc.z, a.Kf, Q.z, Um.z, Uv.z, os);
+                    N.w = outer_elem_adamw(acc.w, a.Kf, Q.w, Um.w, Uv.w, os);
+                    __stcs(reinterpret_cast<float4*>(uv) + i, Uv);
+                } else {
+                    N.x = outer_elem(acc.x, a.Kf, Q.x, Um.x, a.mu, a.lr, a.nesterov);
+                    N.y = outer_elem(acc.y, a.Kf, Q.y, Um.y, a.mu, a.lr, a.nesterov);
+                    N.z = outer_elem(acc.z, a.Kf, Q.z, Um.z, a.mu, a.lr, a.nesterov);
+                    N.w = outer_elem(acc.w, a.Kf, Q.w, Um.w, a.mu, a.lr, a.nesterov);
+                }
                 __stcs(reinterpret_cast<float4*>(xg) + i, N);
                 __stcs(reinterpret_cast<float4*>(um) + i, Um);
                 for (uint32_t k = 0; k < K; ++k) __stcs(reinterpret_cast<float4*>(s_x[k]) + i, N);
@@ -647,8 +670,9 @@ palsgd_outer_kernel(const __grid_constant__ OuterArgs a)
         for (uint32_t i = done + threadIdx.x; i < ch.len; i += kThreads) {
             float sum = s_x[0][i];
             for (uint32_t k = 1; k < K; ++k) sum = __fadd_rn(sum, s_x[k][i]);
-            float ui = um[i];
-            const float xn = outer_elem(sum, a.Kf, xg[i], ui, a.mu, a.lr, a.nesterov);
+            float ui = um[i], xn;
+            if (OOPT) { float vi = uv[i]; xn = outer_elem_adamw(sum, a.Kf, xg[i], ui, vi, os); uv[i] = vi; }
+            else      { xn = outer_elem(sum, a.Kf, xg[i], ui, a.mu, a.lr, a.nesterov); }
             xg[i] = xn; um[i] = ui;
             for (uint32_t k = 0; k < K; ++k) s_x[k][i] = xn;
             if (PREC) { const __nv_bfloat16 h = __float2bfloat16_rn(xn);
@@ -806,7 +830,9 @@ palsgd_init_kernel(const __grid_constant__ OuterArgs a, int has_v)
         const uint32_t seg = ch.seg & ~kSegVecFlag;
         float* xg = tb.global[seg] + ch.off;
         float* um = tb.outer_mom[seg] + ch.off;
+        float* uv = tb.outer_v ? tb.outer_v[seg] + ch.off : nullptr;
         for (uint32_t i = threadIdx.x; i < ch.len; i += kThreads) {
+            if (uv) uv[i] = 0.f;
             float sum = 0.f;
             for (uint32_t k = 0; k < K; ++k) {
                 const size_t pi = (size_t)k * tb.n_seg + seg;

@@ -19,7 +19,9 @@ def cfg_kwargs(cfg) -> dict:
     return dict(K=cfg.K, H=cfg.H, p=cfg.p, inner=cfg.inner, beta1=cfg.beta1, beta2=cfg.beta2,
                 eps=cfg.eps, weight_decay=cfg.weight_decay, momentum=cfg.momentum,
                 outer_lr=cfg.outer_lr, outer_momentum=cfg.outer_momentum,
-                outer_nesterov=cfg.outer_nesterov, seed=cfg.decision_seed, precision=cfg.precision)
+                outer_nesterov=cfg.outer_nesterov, seed=cfg.decision_seed, precision=cfg.precision,
+                outer_opt=cfg.outer_opt, outer_beta1=cfg.outer_beta1, outer_beta2=cfg.outer_beta2,
+                outer_eps=cfg.outer_eps, outer_weight_decay=cfg.outer_weight_decay)
 
 
 def make_oracle(cfg, x0: np.ndarray, dtype: str = "f32") -> oracle.Oracle:
@@ -51,6 +53,8 @@ class GpuRun:
             kinds["v"] = (torch.float32, self.K)
         if self.bf:
             kinds["master"] = (torch.float32, self.K)
+        if cfg.outer_opt == 1:
+            kinds["outer_v"] = (torch.float32, 1)
         self.arena: Dict[str, torch.Tensor] = {}
         self.views: Dict[str, List[List[torch.Tensor]]] = {}
         row = (self.off + self.Ptot + GUARD + 8 + 7) // 8 * 8
@@ -68,7 +72,8 @@ class GpuRun:
         self.stream = torch.cuda.current_stream(self.dev).cuda_stream
         self.lib = P.Palsgd(numel=self.numel, params=v["param"], grads=v["grad"], m=v["m"],
                             v=v.get("v"), master=v.get("master"), global_=v["global_"][0],
-                            outer_mom=v["outer_mom"][0], stream=self.stream, **cfg_kwargs(cfg))
+                            outer_mom=v["outer_mom"][0], outer_v=v["outer_v"][0] if "outer_v" in v else None,
+                            stream=self.stream, **cfg_kwargs(cfg))
 
     # ---- moving data
     def _write(self, name: str, host: np.ndarray) -> None:
@@ -110,6 +115,8 @@ class GpuRun:
             out["v"] = self._read("v")
         if self.bf:
             out["xw"] = self._read("param")
+        if "outer_v" in self.views:
+            out["uv"] = self._read("outer_v")[0]
         return out
 
     def guards_intact(self) -> bool:
@@ -139,6 +146,9 @@ class GpuRun:
     def set_grad_clip(self, max_norm):
         self.lib.set_grad_clip(max_norm)
 
+    def set_outer_lr(self, lr):
+        self.lib.set_outer_lr(lr)
+
     def grad_norms(self):
         return self.lib.get_grad_norms(self.stream)
 
@@ -160,7 +170,7 @@ def ulp_distance(a: np.ndarray, b: np.ndarray) -> int:
 
 
 def compare_state(gpu: Dict[str, np.ndarray], orc: oracle.Oracle, *, rel=REL_TOL, floor=ABS_FLOOR,
-                  names=("x", "m", "v", "xg", "u"), exact: bool = False) -> Dict[str, float]:
+                  names=("x", "m", "v", "xg", "u", "uv"), exact: bool = False) -> Dict[str, float]:
     """Element-by-element comparison.  Returns the worst relative error and ulp
     distance per array; raises on a violation of the tolerance (or of bitwise
     equality when exact=True)."""

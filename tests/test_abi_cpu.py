@@ -31,9 +31,9 @@ def test_library_exports_every_declared_entry_point():
 
 
 def test_config_struct_layout_matches_header():
-    # K, inner, H, eight doubles (p .. outer_momentum), two int32, seed: no padding anywhere
-    assert C.sizeof(B.Config) == 4 + 4 + 8 + 8 * 8 + 4 + 4 + 8 == 96
-    assert B.Config.H.offset == 8 and B.Config.seed.offset == C.sizeof(B.Config) - 8
+    # K, inner, H, eight doubles (p .. outer_momentum), two int32, seed, two int32, four doubles: no padding
+    assert C.sizeof(B.Config) == 4 + 4 + 8 + 8 * 8 + 4 + 4 + 8 + 4 + 4 + 4 * 8 == 136
+    assert B.Config.H.offset == 8 and B.Config.seed.offset == 88 and B.Config.outer_beta1.offset == 104
 
 
 def test_host_decision_matches_oracle_bit_for_bit():

@@ -36,6 +36,11 @@ class WorkloadConfig:
     outer_lr: float = 0.7
     outer_momentum: float = 0.9
     outer_nesterov: bool = True
+    outer_opt: int = 0          # 0 SGD with (Nesterov) momentum, 1 AdamW on the outer gradient
+    outer_beta1: float = 0.9
+    outer_beta2: float = 0.999
+    outer_eps: float = 1e-8
+    outer_weight_decay: float = 0.0
     precision: int = FP32
     init_std: float = 0.02
     grad_std: float = 0.01
