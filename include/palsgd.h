@@ -270,14 +270,19 @@ int palsgd_get_launch_count(palsgd_ctx* ctx, uint64_t* n_launches);
  * CHUNK_MAJOR: order of the (chunk, worker) work items of the register-path inner
  * kernel: 0 = worker index fastest (default), 1 = chunk index fastest.
  * OUTER_SUB_ELEMS: elements per work item of the outer kernel (a slice of a chunk),
- * a multiple of 1024; default 1024.
- * DDP_SUB_ELEMS: the same for the DDP warm-up kernel; default 2048.
+ * a multiple of 1024; default 1024 (4096 for K < 8).
+ * DDP_SUB_ELEMS: the same for the DDP warm-up kernel; default 2048 (4096 in BF16_MASTER mode).
+ * DDP_VARIANT: how the DDP warm-up kernel writes its result to the K slots: 1 = 128-bit stores
+ * by every thread, 2 = staged in shared memory and fanned out by bulk asynchronous stores;
+ * 0 = the library's default (2).
+ * OUTER_VARIANT: the same choice for the outer-sync kernel.
  * (Environment variable PALSGD_CHUNK_ELEMS, read by palsgd_init: elements per chunk
  * = per work item of the inner kernel, a multiple of 1024; default 4096 for fp32 AdamW,
  * 8192 otherwise.) */
 enum { PALSGD_TUNE_INNER_GRID_CAP = 0, PALSGD_TUNE_OUTER_GRID_CAP = 1, PALSGD_TUNE_INNER_VARIANT = 2,
        PALSGD_TUNE_PIPE_STAGES = 3, PALSGD_TUNE_CHUNK_MAJOR = 4, PALSGD_TUNE_OUTER_SUB_ELEMS = 5,
-       PALSGD_TUNE_DDP_SUB_ELEMS = 6 };
+       PALSGD_TUNE_DDP_SUB_ELEMS = 6, PALSGD_TUNE_DDP_VARIANT = 7,
+       PALSGD_TUNE_OUTER_VARIANT = 8 };
 int palsgd_set_tuning(palsgd_ctx* ctx, int knob, int64_t value);
 
 /* The branch draw as a pure host function: 1 = pseudo-sync, 0 = gradient step;

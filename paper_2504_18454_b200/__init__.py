@@ -29,4 +29,6 @@ from .binding import (  # noqa: F401
     TUNE_CHUNK_MAJOR,
     TUNE_OUTER_SUB_ELEMS,
     TUNE_DDP_SUB_ELEMS,
+    TUNE_DDP_VARIANT,
+    TUNE_OUTER_VARIANT,
 )

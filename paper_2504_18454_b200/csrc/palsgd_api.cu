@@ -50,6 +50,8 @@ struct palsgd_ctx {
     uint32_t chunk_elems = kChunkElems;           // elements per chunk-table entry (fixed at init)
     uint32_t outer_sub_elems = kOuterSubElems;    // elements per work item of the outer kernel
     uint32_t ddp_sub_elems = kDdpSubElems;        // elements per work item of the DDP warm-up kernel
+    int ddp_variant = 0;                          // 0 = default, 1 = per-thread stores, 2 = staged bulk stores
+    int outer_variant = 0;                        // the same for the outer kernel
     double max_grad_norm = 0.0;                   // global-norm clip threshold, 0 = off
     double outer_lr = 0.0;                        // OuterOPT learning rate of the next sync
     double opow1 = 1.0, opow2 = 1.0;              // outer_beta^n_outer (AdamW as OuterOPT), running products
@@ -331,6 +333,10 @@ extern "C" int palsgd_init(palsgd_ctx** out, const palsgd_config* cfg, size_t n_
     ctx->P = P;
     ctx->thr = threshold_of(cfg->p);
     ctx->outer_lr = cfg->outer_lr;
+    // work item of the outer kernel, measured on B200: with K + 2 streams per element few slots need
+    // larger slices to amortise the per-item prologue (K = 4: 0.88 -> 0.95 of the copy rate)
+    ctx->outer_sub_elems = K < 8 ? 4096u : kOuterSubElems;
+    ctx->ddp_sub_elems = bf ? 4096u : kDdpSubElems;
     ctx->h_grad_dev.assign(bufs->grad, bufs->grad + (size_t)K * n_tensors);
     ctx->h_global_dev.assign(bufs->global, bufs->global + n_tensors);
 
@@ -541,12 +547,18 @@ extern "C" int palsgd_ddp_step(palsgd_ctx* ctx, double lr_t, void* stream)
     a.clip_on = ctx->max_grad_norm > 0.0 ? 1u : 0u;
     int rc = PALSGD_OK;
     if (a.clip_on) { rc = launch_gradnorm(ctx, true, s); if (rc) return rc; }
-    rc = launch_checked(ctx, [&] {
-        if (adam && !bf)       palsgd_ddp_kernel<0, 0><<<grid, kThreads, 0, s>>>(a);
-        else if (!adam && !bf) palsgd_ddp_kernel<1, 0><<<grid, kThreads, 0, s>>>(a);
-        else if (adam && bf)   palsgd_ddp_kernel<0, 1><<<grid, kThreads, 0, s>>>(a);
-        else                   palsgd_ddp_kernel<1, 1><<<grid, kThreads, 0, s>>>(a);
-    });
+    // staged form: new state in shared memory, fanned out to the K slots by bulk asynchronous stores
+    const size_t stage_bytes = (size_t)a.sub_elems * ((adam ? 12u : 8u) + (bf ? 2u : 0u));
+    const bool bcast = ctx->ddp_variant != 1 && (int)stage_bytes <= ctx->smem_optin - 4096;   // measured best
+    using DdpKernel = void (*)(const DdpArgs);
+    DdpKernel kernel;
+    if (bcast) kernel = adam ? (bf ? palsgd_ddp_kernel<0, 1, 1> : palsgd_ddp_kernel<0, 0, 1>)
+                             : (bf ? palsgd_ddp_kernel<1, 1, 1> : palsgd_ddp_kernel<1, 0, 1>);
+    else       kernel = adam ? (bf ? palsgd_ddp_kernel<0, 1, 0> : palsgd_ddp_kernel<0, 0, 0>)
+                             : (bf ? palsgd_ddp_kernel<1, 1, 0> : palsgd_ddp_kernel<1, 0, 0>);
+    if (bcast && stage_bytes + 4096 > 48 * 1024)   // static + dynamic above the default limit: opt in (idempotent)
+        PALSGD_CUDA(ctx, cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)stage_bytes));
+    rc = launch_checked(ctx, [&] { kernel<<<grid, kThreads, bcast ? stage_bytes : 0, s>>>(a); });
     if (rc) return rc;
     ctx->t += 1;
     return PALSGD_OK;
@@ -580,12 +592,18 @@ extern "C" int palsgd_outer_sync(palsgd_ctx* ctx, void* stream)
         cudaStream_t s = static_cast<cudaStream_t>(stream);
         const bool bf = ctx->cfg.precision == PALSGD_PREC_BF16_MASTER;
         const bool oadam = ctx->cfg.outer_opt == PALSGD_OUTER_ADAMW;
-        int rc = launch_checked(ctx, [&] {
-            if (bf && oadam)       palsgd_outer_kernel<1, 1><<<grid, kThreads, 0, s>>>(a);
-            else if (bf)           palsgd_outer_kernel<1, 0><<<grid, kThreads, 0, s>>>(a);
-            else if (oadam)        palsgd_outer_kernel<0, 1><<<grid, kThreads, 0, s>>>(a);
-            else                   palsgd_outer_kernel<0, 0><<<grid, kThreads, 0, s>>>(a);
-        });
+        // staged form: new x_g (and u, bf16 copy) in shared memory, K slots written by bulk asynchronous stores
+        const size_t stage_bytes = (size_t)a.sub_elems * (8u + (oadam ? 4u : 0u) + (bf ? 2u : 0u));
+        const bool bcast = ctx->outer_variant != 1 && (int)stage_bytes <= ctx->smem_optin - 4096;   // measured best
+        using OuterKernel = void (*)(const OuterArgs);
+        OuterKernel kernel;
+        if (bcast) kernel = bf ? (oadam ? palsgd_outer_kernel<1, 1, 1> : palsgd_outer_kernel<1, 0, 1>)
+                               : (oadam ? palsgd_outer_kernel<0, 1, 1> : palsgd_outer_kernel<0, 0, 1>);
+        else       kernel = bf ? (oadam ? palsgd_outer_kernel<1, 1, 0> : palsgd_outer_kernel<1, 0, 0>)
+                               : (oadam ? palsgd_outer_kernel<0, 1, 0> : palsgd_outer_kernel<0, 0, 0>);
+        if (bcast && stage_bytes + 4096 > 48 * 1024)
+            PALSGD_CUDA(ctx, cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)stage_bytes));
+        int rc = launch_checked(ctx, [&] { kernel<<<grid, kThreads, bcast ? stage_bytes : 0, s>>>(a); });
         if (rc) return rc;
     }
     if (ctx->cfg.outer_opt == PALSGD_OUTER_ADAMW) {
@@ -777,6 +795,14 @@ extern "C" int palsgd_set_tuning(palsgd_ctx* ctx, int knob, int64_t value)
         case PALSGD_TUNE_OUTER_SUB_ELEMS:
             if (value < 1024 || value % 1024 != 0) return PALSGD_EINVAL;
             ctx->outer_sub_elems = (uint32_t)value;
+            return PALSGD_OK;
+        case PALSGD_TUNE_OUTER_VARIANT:
+            if (value > 2) return PALSGD_EINVAL;
+            ctx->outer_variant = (int)value;
+            return PALSGD_OK;
+        case PALSGD_TUNE_DDP_VARIANT:
+            if (value > 2) return PALSGD_EINVAL;
+            ctx->ddp_variant = (int)value;
             return PALSGD_OK;
         case PALSGD_TUNE_DDP_SUB_ELEMS:
             if (value < 1024 || value % 1024 != 0) return PALSGD_EINVAL;

@@ -11,8 +11,8 @@ constexpr uint32_t kThreads     = 256;     // threads per CTA of every kernel he
 constexpr uint32_t kChunkElems  = 8192;    // default elements per chunk-table entry = one work item of the
                                            // inner kernel (large: amortises the per-CTA prologue and tick)
 constexpr uint32_t kStageElems  = 4096;    // stage size of the shared-memory-ring kernels
-constexpr uint32_t kOuterSubElems = 1024;  // default work item of the outer kernel: a slice of a chunk (small:
-                                           // K+2 streams per element need many CTAs in flight)
+constexpr uint32_t kOuterSubElems = 1024;  // default work item of the outer kernel for K >= 8: a slice of a
+                                           // chunk (small: K+2 streams per element need many CTAs in flight)
 constexpr uint32_t kDdpSubElems = 2048;    // default work item of the DDP warm-up kernel (measured)
 constexpr uint32_t kSegVecFlag  = 0x80000000u;   // Chunk::seg bit: 16-byte vector path allowed
 

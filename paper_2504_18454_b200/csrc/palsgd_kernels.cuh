@@ -567,6 +567,24 @@ palsgd_pull_kernel(const __grid_constant__ PullArgs a)
     }
 }
 
+// ---------------------------------------------------------------- bulk stores (TMA engine)
+// One result written to K slots: the CTA stages it in shared memory once and a bulk
+// asynchronous copy per slot and stream (cp.async.bulk shared -> global; this GPU's own
+// memory, no multicast) carries it out, instead of K x 128-bit stores per thread.
+__device__ __forceinline__ void bulk_store(void* dst_gmem, const void* src_smem, uint32_t bytes)
+{
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                 ::"l"(__cvta_generic_to_global(dst_gmem)), "r"((uint32_t)__cvta_generic_to_shared(src_smem)), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_store_commit_and_wait_read()
+{
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+    asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");     // shared memory may be reused after this
+}
+// generic-proxy writes to shared memory become visible to the asynchronous proxy
+__device__ __forceinline__ void fence_async_shared() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
 // ---------------------------------------------------------------- outer sync
 // Per element: average of the K slots in ascending k, outer gradient, (Nesterov)
 // momentum update, and the new global model written to x_g and to all K slots
@@ -592,10 +610,14 @@ __device__ __forceinline__ float outer_elem_adamw(float sum, float Kf, float xg,
 }
 
 // OOPT: 0 = SGD with (Nesterov) momentum, 1 = AdamW (one more state stream).
-template <int PREC, int OOPT>
+// BCAST = 1: the new global model of a work item (and its bf16 copy) is staged in dynamic shared
+// memory (4 + 2 bytes per element, sub_elems elements) and written to the K slots by bulk
+// asynchronous stores; 16-byte-aligned segments only, the rest takes the register path.
+template <int PREC, int OOPT, int BCAST>
 __global__ void __launch_bounds__(kThreads)
 palsgd_outer_kernel(const __grid_constant__ OuterArgs a)
 {
+    extern __shared__ __align__(128) unsigned char outer_stage[];
     const AdamScalars os{a.ob1, a.ob2, a.oomb1, a.oomb2, a.obc1, a.obc2, a.odecay, a.lr, a.oeps};
     __shared__ float* s_x[kMaxWorkers];
     __shared__ __nv_bfloat16* s_w[kMaxWorkers];
@@ -650,13 +672,26 @@ palsgd_outer_kernel(const __grid_constant__ OuterArgs a)
                     N.y = outer_elem_adamw(acc.y, a.Kf, Q.y, Um.y, Uv.y, os);
                     N.z = outer_elem_adamw(acc.z, a.Kf, Q.z, Um.z, Uv.z, os);
                     N.w = outer_elem_adamw(acc.w, a.Kf, Q.w, Um.w, Uv.w, os);
-                    __stcs(reinterpret_cast<float4*>(uv) + i, Uv);
                 } else {
                     N.x = outer_elem(acc.x, a.Kf, Q.x, Um.x, a.mu, a.lr, a.nesterov);
                     N.y = outer_elem(acc.y, a.Kf, Q.y, Um.y, a.mu, a.lr, a.nesterov);
                     N.z = outer_elem(acc.z, a.Kf, Q.z, Um.z, a.mu, a.lr, a.nesterov);
                     N.w = outer_elem(acc.w, a.Kf, Q.w, Um.w, a.mu, a.lr, a.nesterov);
                 }
+                if (BCAST) {
+                    // x_g and u have one destination each and are written once the fan-out below has
+                    // been fixed (a group of 4 left over by the bf16 16-byte rule is redone by the
+                    // scalar loop from unmodified inputs), so they are staged too
+                    float* sx = reinterpret_cast<float*>(outer_stage);
+                    float* su = sx + a.sub_elems;
+                    reinterpret_cast<float4*>(sx)[i] = N;
+                    reinterpret_cast<float4*>(su)[i] = Um;
+                    if (OOPT) reinterpret_cast<float4*>(su + a.sub_elems)[i] = Uv;
+                    if (PREC) reinterpret_cast<uint2*>(su + (OOPT ? 2 : 1) * a.sub_elems)[i] =
+                                  make_uint2(pack_bf16x2(N.x, N.y), pack_bf16x2(N.z, N.w));
+                    continue;
+                }
+                if (OOPT) __stcs(reinterpret_cast<float4*>(uv) + i, Uv);
                 __stcs(reinterpret_cast<float4*>(xg) + i, N);
                 __stcs(reinterpret_cast<float4*>(um) + i, Um);
                 for (uint32_t k = 0; k < K; ++k) __stcs(reinterpret_cast<float4*>(s_x[k]) + i, N);
@@ -666,6 +701,26 @@ palsgd_outer_kernel(const __grid_constant__ OuterArgs a)
                 }
             }
             done = n4 << 2;
+            if (BCAST) {
+                const uint32_t lenb = PREC ? (done & ~7u) : done;       // whole 16-byte units of every stream
+                fence_async_shared();
+                __syncthreads();
+                if (lenb > 0 && threadIdx.x <= K) {
+                    const float* sx = reinterpret_cast<const float*>(outer_stage);
+                    const float* su = sx + a.sub_elems;
+                    if (threadIdx.x == K) {
+                        bulk_store(xg, sx, lenb * 4);
+                        bulk_store(um, su, lenb * 4);
+                        if (OOPT) bulk_store(uv, su + a.sub_elems, lenb * 4);
+                    } else {
+                        bulk_store(s_x[threadIdx.x], sx, lenb * 4);
+                        if (PREC) bulk_store(s_w[threadIdx.x], su + (OOPT ? 2 : 1) * a.sub_elems, lenb * 2);
+                    }
+                    bulk_store_commit_and_wait_read();
+                }
+                done = lenb;
+                __syncthreads();                             // the stage may be overwritten by the next item
+            }
         }
         for (uint32_t i = done + threadIdx.x; i < ch.len; i += kThreads) {
             float sum = s_x[0][i];
@@ -689,10 +744,14 @@ palsgd_outer_kernel(const __grid_constant__ OuterArgs a)
 // gradients) and writes 12K+4 (14K+4) per parameter for AdamW: store-dominated, so the
 // work item is a small slice of a chunk, as in the outer kernel.
 
-template <int INNER, int PREC>
+// BCAST = 1: the new x, m, v (and bf16 copy) of a work item are staged in dynamic shared memory
+// ((12 or 8) + 2 bytes per element, sub_elems elements) and written to the K slots and to x_g
+// by bulk asynchronous stores; 16-byte-aligned segments only, the rest takes the register path.
+template <int INNER, int PREC, int BCAST>
 __global__ void __launch_bounds__(kThreads)
 palsgd_ddp_kernel(const __grid_constant__ DdpArgs a)
 {
+    extern __shared__ __align__(128) unsigned char ddp_stage[];
     __shared__ float* s_x[kMaxWorkers];
     __shared__ float* s_m[kMaxWorkers];
     __shared__ float* s_v[kMaxWorkers];
@@ -765,6 +824,16 @@ palsgd_ddp_kernel(const __grid_constant__ DdpArgs a)
                 G.z = __fdiv_rn(acc.z, a.Kf); G.w = __fdiv_rn(acc.w, a.Kf);
                 if (INNER == 0) { PALSGD_FOR4(adamw_elem(compv(G, c), comp(X, c), comp(M, c), comp(V, c), as)) }
                 else            { PALSGD_FOR4(sgdm_elem(compv(G, c), comp(X, c), comp(M, c), ss)) }
+                if (BCAST) {                                // stage; the fan-out follows the loop
+                    float* sx = reinterpret_cast<float*>(ddp_stage);
+                    float* sm = sx + a.sub_elems;
+                    float* sv = sm + a.sub_elems;
+                    reinterpret_cast<float4*>(sx)[i] = X;
+                    reinterpret_cast<float4*>(sm)[i] = M;
+                    if (INNER == 0) reinterpret_cast<float4*>(sv)[i] = V;
+                    if (PREC) reinterpret_cast<uint2*>(sm + (INNER == 0 ? 2 : 1) * a.sub_elems)[i] = pack4(X);
+                    continue;
+                }
                 __stcs(reinterpret_cast<float4*>(xg) + i, X);
                 for (uint32_t k = 0; k < K; ++k) {
                     __stcs(reinterpret_cast<float4*>(s_x[k]) + i, X);
@@ -777,6 +846,30 @@ palsgd_ddp_kernel(const __grid_constant__ DdpArgs a)
                 }
             }
             done = n4 << 2;
+            if (BCAST) {
+                // whole 16-byte units only: the bf16 stream needs a multiple of 8 elements; what is left
+                // of an odd group of 4 is redone below by the scalar loop (its inputs are still intact)
+                const uint32_t lenb = PREC ? (done & ~7u) : done;
+                fence_async_shared();
+                __syncthreads();
+                if (lenb > 0 && threadIdx.x <= K) {
+                    const float* sx = reinterpret_cast<const float*>(ddp_stage);
+                    const float* sm = sx + a.sub_elems;
+                    const float* sv = sm + a.sub_elems;
+                    if (threadIdx.x == K) {
+                        bulk_store(xg, sx, lenb * 4);
+                    } else {
+                        const uint32_t k = threadIdx.x;
+                        bulk_store(s_x[k], sx, lenb * 4);
+                        bulk_store(s_m[k], sm, lenb * 4);
+                        if (INNER == 0) bulk_store(s_v[k], sv, lenb * 4);
+                        if (PREC) bulk_store(s_w[k], sm + (INNER == 0 ? 2 : 1) * a.sub_elems, lenb * 2);
+                    }
+                    bulk_store_commit_and_wait_read();
+                }
+                done = lenb;
+                __syncthreads();                             // the stage may be overwritten by the next item
+            }
         }
         for (uint32_t i = done + threadIdx.x; i < ch.len; i += kThreads) {
             float sum = 0.f;

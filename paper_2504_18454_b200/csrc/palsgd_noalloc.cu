@@ -156,8 +156,8 @@ extern "C" int palsgd_outer_sync_noalloc(uint32_t K, int32_t precision, size_t n
     a.parts = (kChunkElems + kOuterSubElems - 1) / kOuterSubElems;
     const uint64_t n_items = (uint64_t)n_chunks * a.parts;
     const unsigned grid = (unsigned)(n_items > 0x7FFFFFFFull ? 0x7FFFFFFFull : n_items);
-    if (bf) palsgd_outer_kernel<1, 0><<<grid, kThreads, 0, s>>>(a);
-    else    palsgd_outer_kernel<0, 0><<<grid, kThreads, 0, s>>>(a);
+    if (bf) palsgd_outer_kernel<1, 0, 0><<<grid, kThreads, 0, s>>>(a);
+    else    palsgd_outer_kernel<0, 0, 0><<<grid, kThreads, 0, s>>>(a);
     if (cudaGetLastError() != cudaSuccess) return PALSGD_ECUDA;
     return PALSGD_OK;
 }

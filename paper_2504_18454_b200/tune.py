@@ -122,11 +122,17 @@ def _child(args) -> None:
               f"bytes, {r[1]:.3f} ms on top of a {r[2]:.3f} ms step", flush=True)
     for sub in args.outer_subs:
         ctx.set_tuning(P.TUNE_OUTER_SUB_ELEMS, sub)
-        r = sorted(time_outer() for _ in range(3))
-        print(f"{cfg.name} chunk={chunk} outer slice={sub}: {r[1]:.0f} GB/s (runs {r[0]:.0f}..{r[2]:.0f})", flush=True)
+        for variant in (1, 2):
+            ctx.set_tuning(P.TUNE_OUTER_VARIANT, variant)
+            r = sorted(time_outer() for _ in range(3))
+            print(f"{cfg.name} chunk={chunk} outer slice={sub} variant={variant}: {r[1]:.0f} GB/s "
+                  f"(runs {r[0]:.0f}..{r[2]:.0f})", flush=True)
         ctx.set_tuning(P.TUNE_DDP_SUB_ELEMS, sub)
-        r = sorted(time_ddp() for _ in range(3))
-        print(f"{cfg.name} chunk={chunk} ddp slice={sub}: {r[1]:.0f} GB/s (runs {r[0]:.0f}..{r[2]:.0f})", flush=True)
+        for variant in (1, 2):
+            ctx.set_tuning(P.TUNE_DDP_VARIANT, variant)
+            r = sorted(time_ddp() for _ in range(3))
+            print(f"{cfg.name} chunk={chunk} ddp slice={sub} variant={variant}: {r[1]:.0f} GB/s "
+                  f"(runs {r[0]:.0f}..{r[2]:.0f})", flush=True)
     ctx.destroy()
 
 

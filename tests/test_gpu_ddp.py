@@ -99,6 +99,25 @@ def test_launch_shape_independence_and_launch_count():
             assert np.array_equal(outs[0][k], o[k]), k
 
 
+@pytest.mark.parametrize("inner,precision", [(0, 0), (1, 0), (0, 1), (1, 1)])
+@pytest.mark.parametrize("variant,sub", [(1, 1024), (2, 1024), (2, 2048), (2, 3072), (2, 8192)])
+def test_every_form_of_the_ddp_kernel_matches_oracle(variant, sub, inner, precision):
+    # variant 2 stages the new state in shared memory and writes the K slots with bulk asynchronous
+    # stores; slices that do not fit the stage fall back to per-thread stores
+    numel = [4096 * 5 + 4, 12, 8192 + 6, 1001]
+    P = sum(numel)
+    cfg = _cfg(K=5, inner=inner, precision=precision, momentum=0.9 if inner else 0.0)
+    for layout, cap in (("arena", 0), ("separate", 3), ("misaligned", 0)):
+        x0 = _x0(cfg.K, P, seed=8)
+        gpu, orc = GpuRun(cfg, x0, numel=numel, layout=layout), make_oracle(cfg, x0)
+        gpu.lib.set_tuning(7, variant); gpu.lib.set_tuning(6, sub); gpu.lib.set_tuning(1, cap)
+        for t in range(4):
+            g = _grads(cfg, P, t)
+            gpu.set_grads(g); gpu.ddp_step(cfg.lr); orc.ddp_step(g, cfg.lr)
+        compare_state(gpu.state(), orc, exact=True)
+        assert gpu.guards_intact()
+
+
 def test_resume_inside_the_warm_up_is_bit_exact():
     numel = [10000]
     cfg = _cfg()

@@ -124,3 +124,23 @@ def test_schedule_value_equals_the_oracle_schedule_on_a_grid():
 def test_schedule_value_rejects_bad_arguments():
     assert np.isnan(P.schedule_value(7, 0, 1, 2, 1.0))
     assert np.isnan(P.schedule_value(0, 0, 1, 2, float("inf")))
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("precision,outer_opt", [(0, 0), (1, 0), (0, 1), (1, 1)])
+@pytest.mark.parametrize("variant,sub", [(1, 1024), (2, 1024), (2, 2048), (2, 4096), (2, 16384)])
+def test_every_form_of_the_outer_kernel_matches_oracle(variant, sub, precision, outer_opt):
+    # variant 2 stages the new global model in shared memory and writes the K slots with bulk
+    # asynchronous stores; odd tails and unaligned segments take the per-thread stores
+    numel = [4096 * 5 + 4, 12, 8192 + 6, 1001]
+    Pn = sum(numel)
+    cfg = _cfg(K=5, H=2, T=6, precision=precision, outer_opt=outer_opt, outer_lr=0.7 if outer_opt == 0 else 0.02)
+    for layout, cap in (("arena", 0), ("separate", 3), ("misaligned", 0)):
+        x0 = _x0(cfg.K, Pn, seed=8)
+        gpu, orc = GpuRun(cfg, x0, numel=numel, layout=layout), make_oracle(cfg, x0)
+        gpu.lib.set_tuning(8, variant); gpu.lib.set_tuning(5, sub); gpu.lib.set_tuning(1, cap)
+        for t in range(cfg.T):
+            g = _grads(cfg, Pn, t)
+            gpu.set_grads(g); gpu.step(cfg.lr, cfg.eta); orc.step(g, cfg.lr, cfg.eta)
+        compare_state(gpu.state(), orc, exact=True)
+        assert gpu.guards_intact()
