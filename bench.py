@@ -54,9 +54,10 @@ def measured_peak_gbs():
 # of the same launch, measured on the 16M-element stand-ins of the same kernels (all-gradient inner
 # launch; outer launch).  Traffic grows in proportion to the elements processed, so the ratio carries
 # over to the full-size launch.  Valid only for the kernel sources with the digest recorded here.
-NCU_TRAFFIC = {"digest": "89d23b06744ff9e3",
-               "inner": {0: 0.985, 1: 0.985},      # by precision: fp32, bf16 + fp32 master
-               "outer": {0: 0.957, 1: 0.964}}
+NCU_TRAFFIC = {"digest": "b970f0adff8ab25a",
+               "inner": {0: 0.989, 1: 0.985},      # by precision: fp32, bf16 + fp32 master
+               "outer": {0: 0.957, 1: 0.964},
+               "ddp": {0: 0.975, 1: 0.975}}
 
 
 def kernel_digest() -> str:
@@ -394,7 +395,8 @@ def run_ours(args, cfg):
                               "achieved": ddp["alg_bytes_per_launch"] / (ddp["avg_ms"] * 1e-3) / 1e9,
                               "peak": peak, "unit": "GB/s",
                               "frac": ddp["alg_bytes_per_launch"] / (ddp["avg_ms"] * 1e-3) / 1e9 / peak,
-                              "traffic": None, "launches": ddp["launches"], "avg_ms": ddp["avg_ms"],
+                              "traffic": ncu_traffic("ddp", cfg.precision, ddp["alg_bytes_per_launch"]),
+                              "launches": ddp["launches"], "avg_ms": ddp["avg_ms"],
                               "alg_bytes_per_launch": ddp["alg_bytes_per_launch"],
                               "params_per_s": Pn / (ddp["avg_ms"] * 1e-3),
                               "note": "timed outside the step loop; not part of value"} if ddp else None),
