@@ -207,6 +207,27 @@ double palsgd_schedule_value(int kind, uint64_t t, uint64_t warmup, uint64_t tot
 int palsgd_step(palsgd_ctx* ctx, double lr_t, double eta_t, void* stream);
 
 /*
+ * One synchronisation cycle of Algorithm 1 -- H iterations of the loop body followed by the
+ * outer sync -- as ONE CUDA graph, for models so small that the launches, not the kernels,
+ * set the pace.  Possible because the kernels take t, s_k and the bias-correction products
+ * from device memory: the H inner launches have identical arguments.
+ * palsgd_cycle_capture records the cycle with the given alpha_t, eta_t (constant over the
+ * cycle), the current outer learning rate, clip threshold and tuning knobs; it runs nothing
+ * and may be called again to replace the recording (e.g. when a schedule moves the rates).
+ * It creates a stream and a graph, so call it outside any capture of the caller's own.
+ * palsgd_cycle_launch enqueues the recorded cycle on `stream`: t += H, n_outer += 1.
+ * Both need t to be a multiple of H (a cycle starts right after a sync, or at t = 0).
+ * Results are bit-identical to H calls of palsgd_step.  The gradient buffers are read by each of
+ * the H steps as they stand on the device at that moment: work that refills them between steps
+ * has to be ordered on the device by the caller (e.g. in a graph of the caller's own, around
+ * individual palsgd_inner_step / palsgd_outer_sync launches, which are capturable too).
+ * Errors: EINVAL; ESTATE (t not a multiple of H; launch without a recording);
+ * EUNSUPPORTED (PALSGD_OUTER_ADAMW, whose scalars change every round; H > 65536); ECUDA.
+ */
+int palsgd_cycle_capture(palsgd_ctx* ctx, double lr_t, double eta_t);
+int palsgd_cycle_launch(palsgd_ctx* ctx, void* stream);
+
+/*
  * palsgd_step with HOST gradients and HOST results (the end-to-end call):
  * copies h_grad[k*n_tensors+j] (host, numel[j] elements of the gradient type;
  * pinned memory makes the copies asynchronous) into the gradient buffers, runs

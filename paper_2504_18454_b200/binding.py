@@ -59,6 +59,10 @@ def lib() -> C.CDLL:
     L.palsgd_init.argtypes = [C.POINTER(vp), C.POINTER(Config), C.c_size_t, u64p, C.POINTER(Buffers), vp]
     L.palsgd_inner_step.argtypes = [vp, C.c_double, C.c_double, vp]
     L.palsgd_pseudo_sync.argtypes = [vp, C.c_uint64, C.c_double, vp]
+    L.palsgd_cycle_capture.argtypes = [vp, C.c_double, C.c_double]
+    L.palsgd_cycle_capture.restype = C.c_int
+    L.palsgd_cycle_launch.argtypes = [vp, vp]
+    L.palsgd_cycle_launch.restype = C.c_int
     L.palsgd_ddp_step.argtypes = [vp, C.c_double, vp]
     L.palsgd_ddp_step.restype = C.c_int
     L.palsgd_set_outer_lr.argtypes = [vp, C.c_double]
@@ -214,6 +218,12 @@ class Palsgd:
 
     def step(self, lr_t: float, eta_t: float, stream: int = 0) -> None:
         self._check(lib().palsgd_step(self._ctx, lr_t, eta_t, C.c_void_p(stream)), "palsgd_step")
+
+    def cycle_capture(self, lr_t: float, eta_t: float) -> None:
+        self._check(lib().palsgd_cycle_capture(self._ctx, lr_t, eta_t), "palsgd_cycle_capture")
+
+    def cycle_launch(self, stream: int = 0) -> None:
+        self._check(lib().palsgd_cycle_launch(self._ctx, C.c_void_p(stream)), "palsgd_cycle_launch")
 
     def step_host(self, h_grad_ptrs, lr_t: float, eta_t: float, h_global_ptrs=None,
                   h_decisions_ptr: int = 0, stream: int = 0) -> bool:

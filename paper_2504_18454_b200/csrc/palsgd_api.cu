@@ -55,6 +55,8 @@ struct palsgd_ctx {
     double max_grad_norm = 0.0;                   // global-norm clip threshold, 0 = off
     double outer_lr = 0.0;                        // OuterOPT learning rate of the next sync
     double opow1 = 1.0, opow2 = 1.0;              // outer_beta^n_outer (AdamW as OuterOPT), running products
+    cudaGraphExec_t cycle_exec = nullptr;         // captured H-step cycle (palsgd_cycle_capture) or nullptr
+    uint64_t cycle_launches = 0;                  // kernels inside one captured cycle
     int sm_count = 0, smem_optin = 0;             // device attributes read at init
     std::string cuda_err;
 };
@@ -622,6 +624,51 @@ extern "C" int palsgd_step(palsgd_ctx* ctx, double lr_t, double eta_t, void* str
     return rc;
 }
 
+// ------------------------------------------------------------------------- captured cycle
+
+extern "C" int palsgd_cycle_capture(palsgd_ctx* ctx, double lr_t, double eta_t)
+{
+    if (!ctx) return PALSGD_EINVAL;
+    if (!finite_nonneg(lr_t) || !finite_nonneg(eta_t)) return PALSGD_EINVAL;
+    if (ctx->t % ctx->cfg.H != 0) return PALSGD_ESTATE;             // a cycle starts right after a sync
+    if (ctx->cfg.outer_opt == PALSGD_OUTER_ADAMW) return PALSGD_EUNSUPPORTED;   // its scalars change every round
+    if (ctx->cfg.H > (1u << 16)) return PALSGD_EUNSUPPORTED;
+    if (ctx->cycle_exec) { cudaGraphExecDestroy(ctx->cycle_exec); ctx->cycle_exec = nullptr; }
+
+    // Capture on a stream of our own (the caller's may be the legacy default stream, which cannot capture).
+    // Nothing runs during capture, so the host mirrors are put back afterwards.
+    const uint64_t t0 = ctx->t, n0 = ctx->n_outer, l0 = ctx->launches;
+    cudaStream_t cs = nullptr;
+    PALSGD_CUDA(ctx, cudaStreamCreateWithFlags(&cs, cudaStreamNonBlocking));
+    cudaError_t e = cudaStreamBeginCapture(cs, cudaStreamCaptureModeThreadLocal);
+    int rc = PALSGD_OK;
+    if (e == cudaSuccess) {
+        for (uint64_t i = 0; i < ctx->cfg.H && rc == PALSGD_OK; ++i) rc = palsgd_step(ctx, lr_t, eta_t, cs);
+        cudaGraph_t graph = nullptr;
+        e = cudaStreamEndCapture(cs, &graph);                       // also ends a capture that failed midway
+        if (rc == PALSGD_OK && e == cudaSuccess) e = cudaGraphInstantiate(&ctx->cycle_exec, graph, 0);
+        if (graph) cudaGraphDestroy(graph);
+    }
+    ctx->cycle_launches = ctx->launches - l0;
+    ctx->t = t0; ctx->n_outer = n0; ctx->launches = l0;
+    cudaStreamDestroy(cs);
+    if (rc == PALSGD_OK && e != cudaSuccess) rc = cuda_fail(ctx, e, "cycle capture");
+    if (rc != PALSGD_OK && ctx->cycle_exec) { cudaGraphExecDestroy(ctx->cycle_exec); ctx->cycle_exec = nullptr; }
+    if (rc != PALSGD_OK) (void)cudaGetLastError();
+    return rc;
+}
+
+extern "C" int palsgd_cycle_launch(palsgd_ctx* ctx, void* stream)
+{
+    if (!ctx) return PALSGD_EINVAL;
+    if (!ctx->cycle_exec || ctx->t % ctx->cfg.H != 0) return PALSGD_ESTATE;
+    PALSGD_CUDA(ctx, cudaGraphLaunch(ctx->cycle_exec, static_cast<cudaStream_t>(stream)));
+    ctx->t += ctx->cfg.H;
+    ctx->n_outer += 1;
+    ctx->launches += ctx->cycle_launches;
+    return PALSGD_OK;
+}
+
 extern "C" int palsgd_step_host(palsgd_ctx* ctx, const void* const* h_grad, double lr_t, double eta_t,
                                 float* const* h_global, uint8_t* h_decisions, int* synced, void* stream)
 {
@@ -844,6 +891,7 @@ extern "C" const char* palsgd_last_cuda_error(palsgd_ctx* ctx)
 extern "C" void palsgd_destroy(palsgd_ctx* ctx)
 {
     if (!ctx) return;
+    if (ctx->cycle_exec) cudaGraphExecDestroy(ctx->cycle_exec);
     if (ctx->d_blob) cudaFree(ctx->d_blob);
     delete ctx;
 }
