@@ -97,6 +97,23 @@ def outer_bytes_per_param(cfg) -> int:
     return (10 if cfg.precision == 1 else 8) * cfg.K + 16
 
 
+def max_over_ranks(values, world: int, device=None):
+    """Element-wise MAX of a list of floats over all ranks (the timing rule for N > 1: a job is as
+    slow as its slowest rank).  With one rank the list comes back unchanged."""
+    if world <= 1:
+        return [float(v) for v in values]
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([float(v) for v in values], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def whole_job_value(world: int, K: int, P: int, steps: int, ms_total: float) -> float:
+    """Worker-element updates per second of the whole job: every rank updates K*P elements per step."""
+    return world * K * P * steps / (ms_total * 1e-3)
+
+
 class ClockSampler:
     """nvidia-smi clock / throttle sampling while the timed region runs."""
 
@@ -379,15 +396,12 @@ def run_ours(args, cfg):
         ddp = {"avg_ms": ddp_ms, "alg_bytes_per_launch": ddp_bytes_per_param(cfg) * Pn, "launches": 8}
 
     # ---- max over ranks
-    if world > 1:
-        t = torch.tensor([ms_total, e2e["ms"] if e2e else 0.0], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total, ms_e2e_max = float(t[0]), float(t[1])
-        if e2e:
-            e2e["ms"] = ms_e2e_max
+    ms_total, ms_e2e_max = max_over_ranks([ms_total, e2e["ms"] if e2e else 0.0], world, dev)
+    if e2e:
+        e2e["ms"] = ms_e2e_max
     if rank == 0:
         peak, peak_src = measured_peak_gbs()
-        value = world * K * Pn * args.steps / (ms_total * 1e-3)
+        value = whole_job_value(world, K, Pn, args.steps, ms_total)
         inner_gbs = inner_bytes / (inner_ms * 1e-3) / 1e9 if inner_ms else None
         outer_gbs = outer_bytes / (outer_ms * 1e-3) / 1e9 if outer_ms else None
         line = {

@@ -1,0 +1,70 @@
+"""Full-coverage parity at benchmark size: EVERY element of the GPT-Neo-125M-shaped
+workload (K = 8, 125 M parameters, bf16 working copy + fp32 master) over its full
+512-step schedule against the CPU oracle.
+
+Takes several minutes and 25 GB of host memory, so it only runs when
+PALSGD_FULL_COVERAGE=1 is set; the default suite covers the same workload on a
+sample of indices (tests/test_gpu_configs.py).  Gradients are drawn on the device
+by torch's seeded generator (a harness input), copied to the host every step and
+fed to both sides.
+"""
+import os
+import time
+
+import numpy as np
+import pytest
+import torch
+
+import workloads as W
+from _harness import GpuRun, make_oracle
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.skipif(os.environ.get("PALSGD_FULL_COVERAGE") != "1", reason="set PALSGD_FULL_COVERAGE=1 (slow)")
+@pytest.mark.parametrize("name", ["c3_gptneo125m_bf16"])
+def test_every_element_full_schedule(name):
+    import psutil
+    cfg = W.get_config(name)
+    steps = int(os.environ.get("PALSGD_FULL_COVERAGE_STEPS", cfg.T))
+    K, P = cfg.K, cfg.P
+    need = K * P * (12 + 2 + 2 + 2) + 3 * P * 4 + (4 << 30)          # oracle state, gradient staging, slack
+    if psutil.virtual_memory().available < need:
+        pytest.skip(f"needs {need / 2**30:.0f} GiB of host memory")
+    dev = torch.device("cuda:0")
+    x_init = W.init_params_host(cfg.tensors, cfg.param_seed, cfg.init_std)
+    gpu = GpuRun(cfg, np.broadcast_to(x_init, (K, P)))
+    orc = make_oracle(cfg, np.broadcast_to(x_init, (K, P)))
+    gen = torch.Generator(device=dev); gen.manual_seed(cfg.grad_seed)
+    grad_rows = gpu.arena["grad"][:, gpu.off:gpu.off + P]
+    gdt = torch.bfloat16 if cfg.precision == 1 else torch.float32
+    h_grad = torch.empty((K, P), dtype=gdt).pin_memory()
+    t0 = time.time()
+    for t in range(steps):
+        for k in range(K):
+            grad_rows[k].copy_(torch.randn(P, generator=gen, device=dev, dtype=torch.float32).mul_(cfg.grad_std))
+        h_grad.copy_(grad_rows)
+        g = h_grad.view(torch.int16).numpy().view(np.uint16) if cfg.precision == 1 else h_grad.numpy()
+        gpu.step(cfg.lr, cfg.eta)
+        orc.step(g, cfg.lr, cfg.eta)
+        if t % 32 == 31 or t == steps - 1:
+            c = gpu.counters()
+            assert c["t"] == orc.t and c["n_outer"] == orc.n_outer
+            assert c["s"] == [int(v) for v in orc.s] and c["last_b"] == [int(v) for v in orc.last_b]
+            print(f"step {t + 1}/{steps}: counters equal, {time.time() - t0:.0f} s", flush=True)
+    # every element of every array, bit for bit (one array at a time to bound host memory)
+    torch.cuda.synchronize()
+    pairs = [("master" if cfg.precision == 1 else "param", orc.x), ("m", orc.m)]
+    if cfg.inner == 0:
+        pairs.append(("v", orc.v))
+    if cfg.precision == 1:
+        pairs.append(("param", orc.xw))
+    for name_, want in pairs:
+        got = gpu._read(name_)
+        assert np.array_equal(got, np.asarray(want).reshape(got.shape)), name_
+        del got
+    assert np.array_equal(gpu._read("global_")[0], orc.xg)
+    assert np.array_equal(gpu._read("outer_mom")[0], orc.u)
+    assert gpu.guards_intact()
+    print(f"{name}: all {K * P * (4 if cfg.inner == 0 else 3) + 2 * P} state elements bit-identical after {steps} steps "
+          f"({orc.n_outer} outer syncs), {time.time() - t0:.0f} s", flush=True)
