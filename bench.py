@@ -172,8 +172,20 @@ class ClockSampler:
 
 # ----------------------------------------------------------------------------- CPU oracle leg
 
-def time_oracle(cfg, steps: int, P_sample: int, H: int):
-    """The CPU oracle, as it stands, on the first P_sample elements of the workload."""
+def time_oracle(cfg, steps: int, P_sample: int, H: int, threads: int = 0):
+    """The CPU oracle, as it stands, on the first P_sample elements of the workload
+    (threads = 0: every core the process may use)."""
+    import oracle
+    all_threads = oracle.get_threads()
+    if threads:
+        oracle.set_threads(threads)
+    try:
+        return _time_oracle(cfg, steps, P_sample, H)
+    finally:
+        oracle.set_threads(all_threads)
+
+
+def _time_oracle(cfg, steps: int, P_sample: int, H: int):
     import oracle
     K = cfg.K
     x_init = W.init_params_host(W.flat_shape(P_sample), cfg.param_seed, cfg.init_std)
@@ -256,12 +268,20 @@ def run_ours(args, cfg):
     # CPU baseline first (rank 0, single-GPU runs only), before the GPU is busy
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        # a bounded sample: about 10 s on all cores (step count found from a short trial), 3 s on one
         P_s = min(cfg.P, 1 << 21)
-        H_s = 64
-        value, dt, cores, n_outer = time_oracle(cfg, 64, P_s, H_s)
+        rate, _, _, _ = time_oracle(cfg, 8, P_s, cfg.H)
+        n_steps = int(max(16, min(8192, 10.0 * rate / (cfg.K * P_s))))
+        value, dt, cores, n_outer = time_oracle(cfg, n_steps, P_s, cfg.H)
+        P_1 = min(cfg.P, 1 << 18)
+        rate1, _, _, _ = time_oracle(cfg, 4, P_1, cfg.H, threads=1)
+        n_1 = int(max(8, min(8192, 3.0 * rate1 / (cfg.K * P_1))))
+        value1, dt1, _, _ = time_oracle(cfg, n_1, P_1, cfg.H, threads=1)
         cpu_baseline = {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
-                        "sample": f"first {P_s} of {cfg.P} elements per worker, K={cfg.K}, 64 steps incl. "
-                                  f"{n_outer} outer sync, {dt:.1f} s"}
+                        "sample": f"first {P_s} of {cfg.P} elements per worker, K={cfg.K}, {n_steps} steps incl. "
+                                  f"{n_outer} outer syncs (H={cfg.H}), {dt:.1f} s",
+                        "single_thread_value": value1,
+                        "single_thread_sample": f"first {P_1} elements per worker, {n_1} steps, {dt1:.1f} s"}
 
     # ---- buffers: seeded synthetic values, resident in HBM
     K, Pn = cfg.K, cfg.P
