@@ -374,13 +374,15 @@ def run_ours(args, cfg):
         s0 = torch.cuda.Event(enable_timing=True); s1 = torch.cuda.Event(enable_timing=True)
         s0.record()
         syncs = 0
+        copied_workers = 0                                 # pulling workers' gradients are not transferred
         for _ in range(e2e_steps):
+            copied_workers += sum(1 - P.decision(cfg.decision_seed, t_host, k, cfg.p) for k in range(K))
             syncs += int(ctx.step_host(gp, cfg.lr, cfg.eta, xp, h_dec.data_ptr(), stream)); t_host += 1
         s1.record()
         barrier()
         ms_e2e = s0.elapsed_time(s1)
         e2e = {"ms": ms_e2e, "steps": e2e_steps, "syncs": syncs,
-               "h2d": K * Pn * es, "d2h": K + syncs * Pn * 4 / e2e_steps}
+               "h2d": copied_workers * Pn * es / e2e_steps, "d2h": K + syncs * Pn * 4 / e2e_steps}
 
     # ---- one H-step cycle as a single CUDA graph (launch overhead removed), timed on its own
     graph_cycle = None

@@ -235,7 +235,15 @@ int palsgd_cycle_launch(palsgd_ctx* ctx, void* stream);
  * be NULL) and, if this step ended with an outer sync and h_global is not NULL,
  * the new global model to h_global[j] (float, numel[j] each).  *synced (may be
  * NULL) receives 1 if the outer sync ran.  SYNCHRONISES the stream before
- * returning.  Errors: as palsgd_step.
+ * returning.
+ * The gradient of a worker that pulls in this step is not used by Algorithm 1 and is
+ * NOT copied (its device buffer keeps what it held); palsgd_decision tells the caller
+ * beforehand which workers those are, so it need not produce their gradients at all.
+ * The transfer overlaps the arithmetic: the copies run worker by worker on a stream of
+ * the library's own (ordered after the work already enqueued on `stream`), and the part
+ * of the inner step that belongs to worker k is launched when its gradient has arrived
+ * (K launches per step; with gradient clipping on, or K = 1, one launch after all copies).
+ * Errors: as palsgd_step; EINVAL for a NULL gradient pointer of a non-empty tensor.
  */
 int palsgd_step_host(palsgd_ctx* ctx, const void* const* h_grad, double lr_t, double eta_t,
                      float* const* h_global, uint8_t* h_decisions, int* synced, void* stream);

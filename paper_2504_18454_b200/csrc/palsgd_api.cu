@@ -55,6 +55,9 @@ struct palsgd_ctx {
     double max_grad_norm = 0.0;                   // global-norm clip threshold, 0 = off
     double outer_lr = 0.0;                        // OuterOPT learning rate of the next sync
     double opow1 = 1.0, opow2 = 1.0;              // outer_beta^n_outer (AdamW as OuterOPT), running products
+    cudaStream_t copy_stream = nullptr;           // palsgd_step_host: host -> device copies run here ...
+    std::vector<cudaEvent_t> copy_done;           // ... and signal worker k's gradient with copy_done[k]
+    cudaEvent_t copy_may_start = nullptr;         // recorded on the caller's stream before the copies begin
     cudaGraphExec_t cycle_exec = nullptr;         // captured H-step cycle (palsgd_cycle_capture) or nullptr
     uint64_t cycle_launches = 0;                  // kernels inside one captured cycle
     int sm_count = 0, smem_optin = 0;             // device attributes read at init
@@ -256,7 +259,8 @@ int launch_gradnorm(palsgd_ctx* ctx, bool ddp, cudaStream_t s)
 int launch_inner(palsgd_ctx* ctx, const InnerArgs& a, cudaStream_t s)
 {
     // the shared-memory-ring forms do not carry the clip coefficient: clipped steps take the register path
-    if (!a.clip_on && ctx->inner_variant >= 10 && ctx->inner_variant <= 12 && ctx->tb.n_full > 0 &&
+    const bool whole_step = a.k_begin == 0 && a.k_count == ctx->cfg.K && a.tick;
+    if (whole_step && !a.clip_on && ctx->inner_variant >= 10 && ctx->inner_variant <= 12 && ctx->tb.n_full > 0 &&
         ctx->chunk_elems % kStageElems == 0) {
         const bool adam_ = ctx->cfg.inner == PALSGD_INNER_ADAMW;
         const bool bf_ = ctx->cfg.precision == PALSGD_PREC_BF16_MASTER;
@@ -266,7 +270,7 @@ int launch_inner(palsgd_ctx* ctx, const InnerArgs& a, cudaStream_t s)
         if (adam_ && bf_)   return launch_inner_pipe_nc<0, 1>(ctx, v_, a, s);
         return launch_inner_pipe_nc<1, 1>(ctx, v_, a, s);
     }
-    const uint64_t n_items = (uint64_t)ctx->tb.n_chunks * ctx->cfg.K;
+    const uint64_t n_items = (uint64_t)ctx->tb.n_chunks * a.k_count;
     // with nothing to stream a one-CTA launch still advances the counters
     const unsigned grid = grid_for(n_items, ctx->grid_cap_inner);
     const bool adam = ctx->cfg.inner == PALSGD_INNER_ADAMW;
@@ -486,10 +490,9 @@ extern "C" int palsgd_init(palsgd_ctx** out, const palsgd_config* cfg, size_t n_
 
 // ------------------------------------------------------------------------- steps
 
-extern "C" int palsgd_inner_step(palsgd_ctx* ctx, double lr_t, double eta_t, void* stream)
+// Arguments of the fused inner kernel for one whole step (all K workers, counters ticked).
+static InnerArgs inner_args(const palsgd_ctx* ctx, double lr_t, double eta_t)
 {
-    if (!ctx) return PALSGD_EINVAL;
-    if (!finite_nonneg(lr_t) || !finite_nonneg(eta_t)) return PALSGD_EINVAL;
     const palsgd_config& c = ctx->cfg;
     InnerArgs a{};
     a.tb = ctx->tb;
@@ -512,6 +515,17 @@ extern "C" int palsgd_inner_step(palsgd_ctx* ctx, double lr_t, double eta_t, voi
     a.chunk_major = (uint32_t)ctx->chunk_major;
     // clipped gradients: one norm pass first (not needed when every worker pulls)
     a.clip_on = (ctx->max_grad_norm > 0.0 && c.p < 1.0) ? 1u : 0u;
+    a.k_begin = 0;
+    a.k_count = c.K;
+    a.tick = 1;
+    return a;
+}
+
+extern "C" int palsgd_inner_step(palsgd_ctx* ctx, double lr_t, double eta_t, void* stream)
+{
+    if (!ctx) return PALSGD_EINVAL;
+    if (!finite_nonneg(lr_t) || !finite_nonneg(eta_t)) return PALSGD_EINVAL;
+    const InnerArgs a = inner_args(ctx, lr_t, eta_t);
     int rc = PALSGD_OK;
     if (a.clip_on) { rc = launch_gradnorm(ctx, false, static_cast<cudaStream_t>(stream)); if (rc) return rc; }
     rc = launch_inner(ctx, a, static_cast<cudaStream_t>(stream));
@@ -676,15 +690,21 @@ extern "C" int palsgd_step_host(palsgd_ctx* ctx, const void* const* h_grad, doub
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const size_t n = ctx->n_tensors;
     const size_t gs = elem_size_param(ctx->cfg.precision);
-    // host -> device gradients; tensors adjacent on both sides travel as one copy
-    for (uint32_t k = 0; k < ctx->cfg.K; ++k) {
+    if (!finite_nonneg(lr_t) || !finite_nonneg(eta_t)) return PALSGD_EINVAL;
+    const uint32_t K = ctx->cfg.K;
+    for (size_t i = 0; i < (size_t)K * n; ++i)
+        if (!h_grad[i] && ctx->numel[i % n] > 0) return PALSGD_EINVAL;
+    // host -> device gradients of worker k; tensors adjacent on both sides travel as one copy.
+    // A worker that pulls in this step has no use for a gradient (Algorithm 1 takes one branch or the
+    // other), so nothing is transferred for it.
+    auto copy_worker = [&](uint32_t k, cudaStream_t cs) -> int {
+        if (draw_pull(ctx->cfg.seed, ctx->t, k, ctx->thr)) return PALSGD_OK;
         for (const Segment& sg : ctx->segs) {
             size_t j = sg.first_tensor;
             const size_t end = sg.first_tensor + sg.n_tensors;
             while (j < end) {
                 const size_t idx = (size_t)k * n + j;
                 const char* src = static_cast<const char*>(h_grad[idx]);
-                if (!src) return PALSGD_EINVAL;
                 size_t bytes = ctx->numel[j] * gs;
                 size_t j2 = j + 1;
                 while (j2 < end && static_cast<const char*>(h_grad[(size_t)k * n + j2]) == src + bytes) {
@@ -693,13 +713,46 @@ extern "C" int palsgd_step_host(palsgd_ctx* ctx, const void* const* h_grad, doub
                 }
                 if (bytes)
                     PALSGD_CUDA(ctx, cudaMemcpyAsync(const_cast<void*>(ctx->h_grad_dev[idx]), src, bytes,
-                                                     cudaMemcpyHostToDevice, s));
+                                                     cudaMemcpyHostToDevice, cs));
                 j = j2;
             }
         }
+        return PALSGD_OK;
+    };
+    InnerArgs a = inner_args(ctx, lr_t, eta_t);
+    int rc = PALSGD_OK;
+    if (K > 1 && !a.clip_on) {
+        // Worker by worker: the copies run on a stream of the library's own, and the part of the step that
+        // needs worker k's gradient is launched as soon as that gradient has arrived, so the arithmetic
+        // hides behind the transfer of the following workers.  The last launch ticks the counters.
+        if (!ctx->copy_stream) {
+            PALSGD_CUDA(ctx, cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking));
+            PALSGD_CUDA(ctx, cudaEventCreateWithFlags(&ctx->copy_may_start, cudaEventDisableTiming));
+            ctx->copy_done.resize(K, nullptr);
+            for (uint32_t k = 0; k < K; ++k)
+                PALSGD_CUDA(ctx, cudaEventCreateWithFlags(&ctx->copy_done[k], cudaEventDisableTiming));
+        }
+        PALSGD_CUDA(ctx, cudaEventRecord(ctx->copy_may_start, s));          // earlier readers of the gradients
+        PALSGD_CUDA(ctx, cudaStreamWaitEvent(ctx->copy_stream, ctx->copy_may_start, 0));
+        for (uint32_t k = 0; k < K; ++k) {
+            rc = copy_worker(k, ctx->copy_stream);
+            if (rc) return rc;
+            PALSGD_CUDA(ctx, cudaEventRecord(ctx->copy_done[k], ctx->copy_stream));
+        }
+        for (uint32_t k = 0; k < K; ++k) {
+            PALSGD_CUDA(ctx, cudaStreamWaitEvent(s, ctx->copy_done[k], 0));
+            a.k_begin = k;
+            a.k_count = 1;
+            a.tick = k + 1 == K ? 1u : 0u;
+            rc = launch_inner(ctx, a, s);
+            if (rc) return rc;
+        }
+        ctx->t += 1;
+    } else {
+        for (uint32_t k = 0; k < K; ++k) { rc = copy_worker(k, s); if (rc) return rc; }
+        rc = palsgd_inner_step(ctx, lr_t, eta_t, stream);
+        if (rc) return rc;
     }
-    int rc = palsgd_inner_step(ctx, lr_t, eta_t, stream);
-    if (rc) return rc;
     const bool sync_now = ctx->t % ctx->cfg.H == 0;
     if (sync_now) { rc = palsgd_outer_sync(ctx, stream); if (rc) return rc; }
     if (synced) *synced = sync_now ? 1 : 0;
@@ -892,6 +945,9 @@ extern "C" void palsgd_destroy(palsgd_ctx* ctx)
 {
     if (!ctx) return;
     if (ctx->cycle_exec) cudaGraphExecDestroy(ctx->cycle_exec);
+    for (cudaEvent_t e : ctx->copy_done) if (e) cudaEventDestroy(e);
+    if (ctx->copy_may_start) cudaEventDestroy(ctx->copy_may_start);
+    if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
     if (ctx->d_blob) cudaFree(ctx->d_blob);
     delete ctx;
 }

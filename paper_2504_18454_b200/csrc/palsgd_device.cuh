@@ -75,6 +75,9 @@ struct InnerArgs {
     float    mu, wd;       // momentum SGD scalars
     uint32_t chunk_major;  // 0: worker index fastest over work items; 1: chunk index fastest
     uint32_t clip_on;      // 1: scale worker k's gradient by DevState::clip[k]
+    uint32_t k_begin;      // this launch covers workers k_begin .. k_begin + k_count - 1 (default: all K)
+    uint32_t k_count;
+    uint32_t tick;         // 1: the last CTA advances the device counters (the launch that completes a step)
 };
 
 struct PullArgs {

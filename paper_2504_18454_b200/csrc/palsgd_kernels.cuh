@@ -519,10 +519,13 @@ palsgd_inner_kernel(const __grid_constant__ InnerArgs a)
     }
     __syncthreads();
 
-    const uint64_t n_items = (uint64_t)tb.n_chunks * K;
+    // A step may be split into launches over disjoint worker ranges (gradients that arrive from the
+    // host worker by worker); the last of them ticks the counters for all K workers.
+    const uint32_t Kc = a.k_count;
+    const uint64_t n_items = (uint64_t)tb.n_chunks * Kc;
     for (uint64_t item = blockIdx.x; item < n_items; item += gridDim.x) {
-        const uint32_t k = (uint32_t)(a.chunk_major ? item / tb.n_chunks : item % K);
-        const Chunk ch = tb.chunks[a.chunk_major ? item % tb.n_chunks : item / K];
+        const uint32_t k = a.k_begin + (uint32_t)(a.chunk_major ? item / tb.n_chunks : item % Kc);
+        const Chunk ch = tb.chunks[a.chunk_major ? item % tb.n_chunks : item / Kc];
         if (s_pull[k]) {
             pull_item<PREC, U, kThreads>(threadIdx.x, tb, k, ch, a.beta_pull);
         } else {
@@ -534,7 +537,7 @@ palsgd_inner_kernel(const __grid_constant__ InnerArgs a)
 
     // ---- counter tick by the last CTA (all state reads above precede the atomic)
     __syncthreads();
-    if (threadIdx.x == 0) {
+    if (a.tick && threadIdx.x == 0) {
         __threadfence();
         const unsigned int prev = atomicAdd(&st->done, 1u);
         if (prev == gridDim.x - 1) {

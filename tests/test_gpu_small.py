@@ -226,3 +226,30 @@ def test_step_host_moves_gradients_and_results_through_host_buffers():
             if synced:
                 assert np.array_equal(hx.numpy(), orc.xg)
         compare_state(gpu.state(), orc, exact=True)
+
+
+def test_step_host_transfers_no_gradient_for_workers_that_pull_and_splits_the_step_per_worker():
+    numel = [6000, 9]
+    P = sum(numel)
+    cfg = _cfg(numel, K=6, p=0.5, H=100)
+    x0 = _x0(cfg.K, P, same=True)
+    gpu, orc = GpuRun(cfg, x0, numel=numel, layout="arena"), make_oracle(cfg, x0)
+    hg = torch.empty((cfg.K, P), dtype=torch.float32).pin_memory()
+    starts = np.concatenate([[0], np.cumsum(numel)])
+    gp = gpu.lib.make_ptr_array([hg.data_ptr() + (k * P + int(starts[j])) * 4
+                                 for k in range(cfg.K) for j in range(len(numel))])
+    launches = gpu.lib.get_launch_count()
+    for t in range(6):
+        marker = np.full((cfg.K, P), 1000.0 + t, dtype=np.float32)
+        gpu.set_grads(marker)                                     # what the device buffers held before the call
+        g = _grads(cfg, P, t)
+        hg.copy_(torch.from_numpy(g))
+        gpu.lib.step_host(gp, cfg.lr, cfg.eta, None, 0, gpu.stream)
+        orc.step(g, cfg.lr, cfg.eta)
+        on_device = gpu._read("grad")
+        for k in range(cfg.K):
+            want = marker[k] if orc.last_b[k] else g[k]           # pulled: untouched; gradient step: copied
+            assert np.array_equal(on_device[k], want), (t, k)
+    compare_state(gpu.state(), orc, exact=True)
+    assert gpu.lib.get_launch_count() - launches == 6 * cfg.K     # one launch per worker and step
+    assert gpu.counters()["s"] == [int(v) for v in orc.s]
