@@ -220,7 +220,7 @@ def run_reference(args, cfg):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f32" if cfg.precision == 0 else "f32 math, bf16 params/grads",
+        "dtype": "f32",
         "data": "synthetic", "config": workload_config(cfg, args),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -430,7 +430,7 @@ def run_ours(args, cfg):
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_total / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "f32" if cfg.precision == 0 else "f32 math, bf16 params/grads",
+            "dtype": "f32",
             "data": "synthetic", "config": workload_config(cfg, args),
             "roofline": {"bound": "hbm", "kernel": "palsgd_inner_kernel", "achieved": inner_gbs,
                          "peak": peak, "unit": "GB/s", "frac": inner_gbs / peak if inner_gbs else None,
