@@ -119,3 +119,39 @@ def test_missing_library_is_a_loud_error(monkeypatch, tmp_path):
     monkeypatch.setattr(B, "LIB_PATH", tmp_path / "nope.so")
     with pytest.raises(ImportError):
         B.lib()
+
+
+def test_later_entry_points_reject_a_null_context():
+    L = P.lib()
+    assert L.palsgd_ddp_step(None, 1e-3, None) == -1
+    assert L.palsgd_set_grad_clip(None, 1.0) == -1
+    assert L.palsgd_get_grad_norms(None, None, None, None) == -1
+    assert L.palsgd_set_outer_lr(None, 0.5) == -1
+    assert L.palsgd_cycle_capture(None, 1e-3, 1.0) == -1
+    assert L.palsgd_cycle_launch(None, None) == -1
+    assert L.palsgd_step_host(None, None, 1e-3, 1.0, None, None, None, None) == -1
+    assert L.palsgd_set_tuning(None, 0, 0) == -1
+
+
+@pytest.mark.parametrize("over", [dict(outer_opt=2), dict(outer_opt=1),                      # AdamW outer without outer_v
+                                  dict(outer_opt=1, outer_beta1=1.0), dict(outer_opt=1, outer_eps=-1.0)])
+def test_init_rejects_bad_outer_optimizer_settings(over):
+    assert _fake_init(**over) == -1
+
+
+def test_no_allocation_entry_point_validates_before_touching_the_gpu():
+    L = P.lib()
+    vp = C.c_void_p
+    arr = lambda *a: C.cast((vp * len(a))(*[vp(x) for x in a]), C.POINTER(vp))
+    numel = (C.c_uint64 * 1)(8)
+    ok_ptrs = dict(param=arr(0x10000), master=None, global_=arr(0x20000), outer_mom=arr(0x30000))
+    call = lambda K=1, prec=0, numel=numel, lr=0.7, mu=0.9, nest=1, **p: L.palsgd_outer_sync_noalloc(
+        K, prec, 1, numel, p.get("param", ok_ptrs["param"]), p.get("master", None),
+        p.get("global_", ok_ptrs["global_"]), p.get("outer_mom", ok_ptrs["outer_mom"]), lr, mu, nest, None)
+    assert call(K=0) == -1 and call(K=65) == -1 and call(prec=2) == -1 and call(nest=2) == -1
+    assert call(lr=float("nan")) == -1 and call(mu=-0.5) == -1
+    assert call(prec=1) == -1                                            # mixed precision needs the masters
+    assert call(param=arr(0)) == -1                                      # NULL slot pointer of a non-empty tensor
+    assert call(param=arr(0x10002)) == -2                                # not aligned to the element size
+    assert call(numel=(C.c_uint64 * 1)(8192 * 70000)) == -8              # tables beyond the fixed scratch
+    assert call(numel=(C.c_uint64 * 1)(0)) == 0                          # nothing to do
