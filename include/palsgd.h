@@ -291,10 +291,11 @@ int palsgd_get_launch_count(palsgd_ctx* ctx, uint64_t* n_launches);
 /* Launch-shape knobs (advanced; results never depend on them).
  * *_GRID_CAP: the largest grid a launch may use, CTAs looping over work items
  * beyond it; 0 (default) = one CTA per work item.
- * INNER_VARIANT: which compiled form of the fused inner kernel runs: 1..9 =
- * register-path shapes (loads in flight per thread x CTAs per SM), 10 / 11 / 12 = the
- * persistent shared-memory-ring form with 512 / 256 / 1024 consumer threads; 0 = the
- * library's default, unknown = default.
+ * INNER_VARIANT: which form of the fused inner kernel runs: 0 = the library's default (the measured
+ * best launch shape as a persistent grid that draws its work items from a queue in device memory);
+ * 18 = the same shape with one CTA per work item; 1..9, 13..15 = other register-path shapes (loads in
+ * flight per thread x CTAs per SM), one CTA per item; 10 / 11 / 12 = the persistent shared-memory-ring
+ * form with 512 / 256 / 1024 consumer threads; unknown = default.
  * PIPE_STAGES: ring depth of the persistent form; 0 = as many as fit.
  * CHUNK_MAJOR: order of the (chunk, worker) work items of the register-path inner
  * kernel: 0 = worker index fastest (default), 1 = chunk index fastest.
@@ -305,13 +306,16 @@ int palsgd_get_launch_count(palsgd_ctx* ctx, uint64_t* n_launches);
  * by every thread, 2 = staged in shared memory and fanned out by bulk asynchronous stores;
  * 0 = the library's default (2).
  * OUTER_VARIANT: the same choice for the outer-sync kernel.
+ * OUTER_DYNAMIC: outer-sync and DDP kernels as a persistent grid of that many CTAs per SM that
+ * draws its work items from a queue; 0 = one CTA per work item.  Until this knob is set the
+ * library uses its defaults (outer sync: one CTA per item; DDP step: 4 CTAs per SM).
  * (Environment variable PALSGD_CHUNK_ELEMS, read by palsgd_init: elements per chunk
  * = per work item of the inner kernel, a multiple of 1024; default 4096 for fp32 AdamW,
  * 8192 otherwise.) */
 enum { PALSGD_TUNE_INNER_GRID_CAP = 0, PALSGD_TUNE_OUTER_GRID_CAP = 1, PALSGD_TUNE_INNER_VARIANT = 2,
        PALSGD_TUNE_PIPE_STAGES = 3, PALSGD_TUNE_CHUNK_MAJOR = 4, PALSGD_TUNE_OUTER_SUB_ELEMS = 5,
        PALSGD_TUNE_DDP_SUB_ELEMS = 6, PALSGD_TUNE_DDP_VARIANT = 7,
-       PALSGD_TUNE_OUTER_VARIANT = 8 };
+       PALSGD_TUNE_OUTER_VARIANT = 8, PALSGD_TUNE_OUTER_DYNAMIC = 9 };
 int palsgd_set_tuning(palsgd_ctx* ctx, int knob, int64_t value);
 
 /* The branch draw as a pure host function: 1 = pseudo-sync, 0 = gradient step;

@@ -31,4 +31,5 @@ from .binding import (  # noqa: F401
     TUNE_DDP_SUB_ELEMS,
     TUNE_DDP_VARIANT,
     TUNE_OUTER_VARIANT,
+    TUNE_OUTER_DYNAMIC,
 )

@@ -14,7 +14,7 @@ OUTER_SGD, OUTER_ADAMW = 0, 1
 SCHED_WARMUP_CONSTANT, SCHED_WARMUP_COSINE = 0, 1
 TUNE_INNER_GRID_CAP, TUNE_OUTER_GRID_CAP, TUNE_INNER_VARIANT, TUNE_PIPE_STAGES = 0, 1, 2, 3
 TUNE_CHUNK_MAJOR, TUNE_OUTER_SUB_ELEMS, TUNE_DDP_SUB_ELEMS, TUNE_DDP_VARIANT = 4, 5, 6, 7
-TUNE_OUTER_VARIANT = 8
+TUNE_OUTER_VARIANT, TUNE_OUTER_DYNAMIC = 8, 9
 MAX_WORKERS = 64
 
 

@@ -33,6 +33,7 @@ struct DevState {
     unsigned long long s[kMaxWorkers];       // gradient steps taken by worker k
     double             pow1[kMaxWorkers];    // beta1^s_k  (running product, binary64)
     double             pow2[kMaxWorkers];    // beta2^s_k
+    unsigned int       queue;                // next work item of a launch that hands items out dynamically
     unsigned int       done;                 // CTAs that finished the current inner launch
     unsigned int       error;                // 0, or the code of a bounded wait that expired
     unsigned char      last_b[kMaxWorkers];  // decisions of the latest inner step
@@ -78,6 +79,7 @@ struct InnerArgs {
     uint32_t k_begin;      // this launch covers workers k_begin .. k_begin + k_count - 1 (default: all K)
     uint32_t k_count;
     uint32_t tick;         // 1: the last CTA advances the device counters (the launch that completes a step)
+    uint32_t dynamic;      // 1: a persistent grid takes work items from DevState::queue (needs tick = 1)
 };
 
 struct PullArgs {
@@ -93,6 +95,7 @@ struct OuterArgs {
     float  ob1, ob2, oomb1, oomb2, obc1, obc2, odecay, oeps;   // AdamW as OuterOPT (step n_outer + 1)
     uint32_t sub_elems;    // elements per work item (a multiple of 4 * kThreads)
     uint32_t parts;        // work items per chunk = ceil(chunk_elems / sub_elems)
+    uint32_t dynamic;      // 1: a persistent grid takes work items from DevState::queue
 };
 
 // DDP warm-up step: averaged gradient, one optimizer step taken on worker 0's state, written to all.
@@ -106,6 +109,7 @@ struct DdpArgs {
     uint32_t sub_elems;    // elements per work item (a multiple of 4 * kThreads)
     uint32_t parts;        // work items per chunk
     uint32_t clip_on;      // 1: scale the averaged gradient by DevState::clip[0]
+    uint32_t dynamic;      // 1: a persistent grid takes work items from DevState::queue
 };
 
 // Gradient-norm pass of the global-norm clip.

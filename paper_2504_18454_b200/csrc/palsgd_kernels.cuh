@@ -523,7 +523,16 @@ palsgd_inner_kernel(const __grid_constant__ InnerArgs a)
     // host worker by worker); the last of them ticks the counters for all K workers.
     const uint32_t Kc = a.k_count;
     const uint64_t n_items = (uint64_t)tb.n_chunks * Kc;
-    for (uint64_t item = blockIdx.x; item < n_items; item += gridDim.x) {
+    __shared__ unsigned int s_item;
+    // a.dynamic: a grid of a few CTAs per SM draws items from a counter, so no CTA idles while others
+    // still have a backlog; otherwise item = blockIdx.x, strided by the grid
+    uint64_t item = blockIdx.x;
+    if (a.dynamic) {
+        if (threadIdx.x == 0) s_item = atomicAdd(&st->queue, 1u);
+        __syncthreads();
+        item = s_item;
+    }
+    while (item < n_items) {
         const uint32_t k = a.k_begin + (uint32_t)(a.chunk_major ? item / tb.n_chunks : item % Kc);
         const Chunk ch = tb.chunks[a.chunk_major ? item % tb.n_chunks : item / Kc];
         if (s_pull[k]) {
@@ -532,6 +541,14 @@ palsgd_inner_kernel(const __grid_constant__ InnerArgs a)
             const AdamScalars as{a.b1, a.b2, a.omb1, a.omb2, s_bc1[k], s_bc2[k], a.decay, a.lr, a.eps, s_clip[k]};
             const SgdScalars  ss{a.mu, a.wd, a.lr, s_clip[k]};
             grad_item<INNER, PREC, U, kThreads>(threadIdx.x, tb, k, ch, as, ss);
+        }
+        if (a.dynamic) {
+            __syncthreads();                                   // everyone has read s_item
+            if (threadIdx.x == 0) s_item = atomicAdd(&st->queue, 1u);
+            __syncthreads();
+            item = s_item;
+        } else {
+            item += gridDim.x;
         }
     }
 
@@ -551,6 +568,7 @@ palsgd_inner_kernel(const __grid_constant__ InnerArgs a)
             }
             st->t = t + 1;
             st->done = 0;
+            st->queue = 0;                                     // every CTA has drawn its last item by now
             __threadfence();
         }
     }
@@ -567,6 +585,35 @@ palsgd_pull_kernel(const __grid_constant__ PullArgs a)
     for (uint64_t item = blockIdx.x; item < n_items; item += gridDim.x) {
         const uint32_t k = (uint32_t)(item % K);
         if ((a.mask >> k) & 1ull) pull_item<PREC, U, kThreads>(threadIdx.x, tb, k, tb.chunks[item / K], a.beta);
+    }
+}
+
+// ---------------------------------------------------------------- work distribution
+// Next work item of a CTA: strided by the grid, or (dynamic) drawn from a counter in device memory by
+// a persistent grid.  Called by all threads of the CTA; s_item is a shared-memory word of the caller.
+__device__ __forceinline__ uint64_t first_item(uint32_t dynamic, DevState* st, unsigned int* s_item)
+{
+    if (!dynamic) return blockIdx.x;
+    if (threadIdx.x == 0) *s_item = atomicAdd(&st->queue, 1u);
+    __syncthreads();
+    return *s_item;
+}
+__device__ __forceinline__ uint64_t next_item(uint64_t cur, uint32_t dynamic, DevState* st, unsigned int* s_item)
+{
+    if (!dynamic) return cur + gridDim.x;
+    __syncthreads();                                           // everyone has read *s_item
+    if (threadIdx.x == 0) *s_item = atomicAdd(&st->queue, 1u);
+    __syncthreads();
+    return *s_item;
+}
+// After the loop of a dynamic launch: the last CTA to finish rewinds the queue for the next launch.
+__device__ __forceinline__ void rewind_queue(DevState* st)
+{
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        const unsigned int prev = atomicAdd(&st->done, 1u);
+        if (prev == gridDim.x - 1) { st->done = 0; st->queue = 0; __threadfence(); }
     }
 }
 
@@ -628,8 +675,10 @@ palsgd_outer_kernel(const __grid_constant__ OuterArgs a)
     const uint32_t K = tb.K;
     constexpr int B = 8;                                   // slot loads issued together
 
+    __shared__ unsigned int s_item;
     const uint64_t n_items = (uint64_t)tb.n_chunks * a.parts;
-    for (uint64_t item = blockIdx.x; item < n_items; item += gridDim.x) {
+    for (uint64_t item = first_item(a.dynamic, tb.st, &s_item); item < n_items;
+         item = next_item(item, a.dynamic, tb.st, &s_item)) {
         Chunk ch = tb.chunks[item / a.parts];
         const uint32_t begin = (uint32_t)(item % a.parts) * a.sub_elems;      // this item's slice of the chunk
         if (begin >= ch.len) continue;                                        // uniform over the CTA
@@ -737,6 +786,7 @@ palsgd_outer_kernel(const __grid_constant__ OuterArgs a)
                         for (uint32_t k = 0; k < K; ++k) s_w[k][i] = h; }
         }
     }
+    if (a.dynamic) rewind_queue(tb.st);
 }
 
 // ---------------------------------------------------------------- DDP warm-up step
@@ -775,8 +825,10 @@ palsgd_ddp_kernel(const __grid_constant__ DdpArgs a)
     SgdScalars ss{a.mu, a.wd, a.lr};
     if (a.clip_on) { as.clip = st->clip[0]; ss.clip = as.clip; }   // the clip applies to the averaged gradient
 
+    __shared__ unsigned int s_item;
     const uint64_t n_items = (uint64_t)tb.n_chunks * a.parts;
-    for (uint64_t item = blockIdx.x; item < n_items; item += gridDim.x) {
+    for (uint64_t item = first_item(a.dynamic, st, &s_item); item < n_items;
+         item = next_item(item, a.dynamic, st, &s_item)) {
         Chunk ch = tb.chunks[item / a.parts];
         const uint32_t begin = (uint32_t)(item % a.parts) * a.sub_elems;
         if (begin >= ch.len) continue;                                        // uniform over the CTA
@@ -908,6 +960,7 @@ palsgd_ddp_kernel(const __grid_constant__ DdpArgs a)
             }
             st->t = t + 1;
             st->done = 0;
+            st->queue = 0;
             __threadfence();
         }
     }

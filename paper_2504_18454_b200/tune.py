@@ -13,6 +13,7 @@ from __future__ import annotations
 
 import argparse
 import os
+import time
 import subprocess
 import sys
 
@@ -66,6 +67,7 @@ def _child(args) -> None:
         return byts / ms / 1e6
 
     def time_outer(reps=8):
+        heat()
         for _ in range(2):
             ctx.outer_sync(stream)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -77,7 +79,18 @@ def _child(args) -> None:
         per = (10 if cfg.precision == 1 else 8) * cfg.K + 16
         return per * cfg.P / (e0.elapsed_time(e1) / reps) / 1e6
 
+    def heat():
+        # optional: load the GPU for a while first, so that the timing sees the clocks of a long run
+        if args.heat_ms > 0:
+            ctx.set_grad_clip(0.0)
+            t0 = time.time()
+            while (time.time() - t0) * 1e3 < args.heat_ms:
+                for _ in range(16):
+                    ctx.inner_step(cfg.lr, cfg.eta, stream)
+                torch.cuda.synchronize()
+
     def time_ddp(reps=8):
+        heat()
         for _ in range(2):
             ctx.ddp_step(cfg.lr, stream)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -120,7 +133,9 @@ def _child(args) -> None:
         r = sorted(time_norm(args.steps, ddp) for _ in range(3))[1]
         print(f"{cfg.name} chunk={chunk} grad-norm pass ({'ddp' if ddp else 'per worker'}): {r[0]:.0f} GB/s of gradient "
               f"bytes, {r[1]:.3f} ms on top of a {r[2]:.3f} ms step", flush=True)
-    for sub in args.outer_subs:
+    for sub, dyn in [(s_, d_) for s_ in args.outer_subs for d_ in args.outer_dynamic]:
+        ctx.set_tuning(P.TUNE_OUTER_DYNAMIC, dyn)
+        chunk = f"{os.environ.get('PALSGD_CHUNK_ELEMS', 'default')} dyn={dyn}"
         ctx.set_tuning(P.TUNE_OUTER_SUB_ELEMS, sub)
         for variant in (1, 2):
             ctx.set_tuning(P.TUNE_OUTER_VARIANT, variant)
@@ -143,7 +158,10 @@ def main() -> None:
     ap.add_argument("--variants", type=ints, default=[0])
     ap.add_argument("--chunks", type=ints, default=[])
     ap.add_argument("--outer-subs", type=ints, default=[1024])
+    ap.add_argument("--outer-dynamic", type=ints, default=[0], help="CTAs per SM of the persistent outer/DDP grid; 0 = off")
     ap.add_argument("--steps", type=int, default=40)
+    ap.add_argument("--heat-ms", type=float, default=0.0,
+                    help="run inner steps for this long before each outer/DDP timing (power-capped clocks)")
     ap.add_argument("--child", action="store_true", help=argparse.SUPPRESS)
     args = ap.parse_args()
     if args.child or not args.chunks:
@@ -153,7 +171,8 @@ def main() -> None:
         env = dict(os.environ, PALSGD_CHUNK_ELEMS=str(ce))
         cmd = [sys.executable, "-m", "paper_2504_18454_b200.tune", args.workload, "--child",
                "--variants", ",".join(map(str, args.variants)),
-               "--outer-subs", ",".join(map(str, args.outer_subs)), "--steps", str(args.steps)]
+               "--outer-subs", ",".join(map(str, args.outer_subs)), "--steps", str(args.steps),
+               "--outer-dynamic", ",".join(map(str, args.outer_dynamic)), "--heat-ms", str(args.heat_ms)]
         subprocess.run(cmd, env=env, check=True, cwd=ROOT)
 
 

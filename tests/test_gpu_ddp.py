@@ -100,8 +100,9 @@ def test_launch_shape_independence_and_launch_count():
 
 
 @pytest.mark.parametrize("inner,precision", [(0, 0), (1, 0), (0, 1), (1, 1)])
-@pytest.mark.parametrize("variant,sub", [(1, 1024), (2, 1024), (2, 2048), (2, 3072), (2, 8192)])
-def test_every_form_of_the_ddp_kernel_matches_oracle(variant, sub, inner, precision):
+@pytest.mark.parametrize("variant,sub,dyn", [(1, 1024, 0), (2, 1024, 0), (2, 2048, 0), (2, 3072, 0), (2, 8192, 0),
+                                             (1, 1024, 3), (2, 2048, 2)])
+def test_every_form_of_the_ddp_kernel_matches_oracle(variant, sub, dyn, inner, precision):
     # variant 2 stages the new state in shared memory and writes the K slots with bulk asynchronous
     # stores; slices that do not fit the stage fall back to per-thread stores
     numel = [4096 * 5 + 4, 12, 8192 + 6, 1001]
@@ -111,6 +112,7 @@ def test_every_form_of_the_ddp_kernel_matches_oracle(variant, sub, inner, precis
         x0 = _x0(cfg.K, P, seed=8)
         gpu, orc = GpuRun(cfg, x0, numel=numel, layout=layout), make_oracle(cfg, x0)
         gpu.lib.set_tuning(7, variant); gpu.lib.set_tuning(6, sub); gpu.lib.set_tuning(1, cap)
+        gpu.lib.set_tuning(9, dyn)                    # persistent grid + work queue (ignored when the grid is capped)
         for t in range(4):
             g = _grads(cfg, P, t)
             gpu.set_grads(g); gpu.ddp_step(cfg.lr); orc.ddp_step(g, cfg.lr)

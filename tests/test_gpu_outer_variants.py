@@ -128,8 +128,9 @@ def test_schedule_value_rejects_bad_arguments():
 
 @pytest.mark.gpu
 @pytest.mark.parametrize("precision,outer_opt", [(0, 0), (1, 0), (0, 1), (1, 1)])
-@pytest.mark.parametrize("variant,sub", [(1, 1024), (2, 1024), (2, 2048), (2, 4096), (2, 16384)])
-def test_every_form_of_the_outer_kernel_matches_oracle(variant, sub, precision, outer_opt):
+@pytest.mark.parametrize("variant,sub,dyn", [(1, 1024, 0), (2, 1024, 0), (2, 2048, 0), (2, 4096, 0), (2, 16384, 0),
+                                             (1, 1024, 2), (2, 1024, 4), (2, 4096, 1)])
+def test_every_form_of_the_outer_kernel_matches_oracle(variant, sub, dyn, precision, outer_opt):
     # variant 2 stages the new global model in shared memory and writes the K slots with bulk
     # asynchronous stores; odd tails and unaligned segments take the per-thread stores
     numel = [4096 * 5 + 4, 12, 8192 + 6, 1001]
@@ -139,6 +140,7 @@ def test_every_form_of_the_outer_kernel_matches_oracle(variant, sub, precision, 
         x0 = _x0(cfg.K, Pn, seed=8)
         gpu, orc = GpuRun(cfg, x0, numel=numel, layout=layout), make_oracle(cfg, x0)
         gpu.lib.set_tuning(8, variant); gpu.lib.set_tuning(5, sub); gpu.lib.set_tuning(1, cap)
+        gpu.lib.set_tuning(9, dyn)                    # persistent grid + work queue (ignored when the grid is capped)
         for t in range(cfg.T):
             g = _grads(cfg, Pn, t)
             gpu.set_grads(g); gpu.step(cfg.lr, cfg.eta); orc.step(g, cfg.lr, cfg.eta)

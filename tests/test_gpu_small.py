@@ -179,7 +179,7 @@ def test_run_to_run_determinism_and_launch_shape_independence():
 
 
 @pytest.mark.parametrize("variant,stages,cap", [(10, 0, 0), (11, 0, 0), (12, 0, 0), (10, 2, 3), (11, 3, 1), (12, 2, 2),
-                                                (3, 0, 0), (5, 0, 5), (7, 0, 0), (9, 0, 0), (13, 0, 0), (15, 0, 9)])
+                                                (3, 0, 0), (5, 0, 5), (7, 0, 0), (9, 0, 0), (13, 0, 0), (15, 0, 9), (18, 0, 0), (18, 0, 7)])
 @pytest.mark.parametrize("inner,precision", [(0, 0), (1, 0), (0, 1), (1, 1)])
 def test_every_compiled_form_of_the_inner_kernel_matches_oracle(variant, stages, cap, inner, precision):
     # 10/11: persistent shared-memory-ring form (full chunks through the ring, the rest by registers)
