@@ -238,12 +238,14 @@ int palsgd_cycle_launch(palsgd_ctx* ctx, void* stream);
  * returning.
  * The gradient of a worker that pulls in this step is not used by Algorithm 1 and is
  * NOT copied (its device buffer keeps what it held); palsgd_decision tells the caller
- * beforehand which workers those are, so it need not produce their gradients at all.
+ * beforehand which workers those are, so it need not produce their gradients at all
+ * (their h_grad entries may be NULL).
  * The transfer overlaps the arithmetic: the copies run worker by worker on a stream of
  * the library's own (ordered after the work already enqueued on `stream`), and the part
  * of the inner step that belongs to worker k is launched when its gradient has arrived
  * (K launches per step; with gradient clipping on, or K = 1, one launch after all copies).
- * Errors: as palsgd_step; EINVAL for a NULL gradient pointer of a non-empty tensor.
+ * Errors: as palsgd_step; EINVAL for a NULL gradient pointer of a non-empty tensor of a
+ * worker that takes a gradient step.
  */
 int palsgd_step_host(palsgd_ctx* ctx, const void* const* h_grad, double lr_t, double eta_t,
                      float* const* h_global, uint8_t* h_decisions, int* synced, void* stream);

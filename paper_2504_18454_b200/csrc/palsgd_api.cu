@@ -716,8 +716,11 @@ extern "C" int palsgd_step_host(palsgd_ctx* ctx, const void* const* h_grad, doub
     const size_t gs = elem_size_param(ctx->cfg.precision);
     if (!finite_nonneg(lr_t) || !finite_nonneg(eta_t)) return PALSGD_EINVAL;
     const uint32_t K = ctx->cfg.K;
-    for (size_t i = 0; i < (size_t)K * n; ++i)
-        if (!h_grad[i] && ctx->numel[i % n] > 0) return PALSGD_EINVAL;
+    for (uint32_t k = 0; k < K; ++k) {                       // a pulling worker's pointers are not looked at
+        if (draw_pull(ctx->cfg.seed, ctx->t, k, ctx->thr)) continue;
+        for (size_t j = 0; j < n; ++j)
+            if (!h_grad[(size_t)k * n + j] && ctx->numel[j] > 0) return PALSGD_EINVAL;
+    }
     // host -> device gradients of worker k; tensors adjacent on both sides travel as one copy.
     // A worker that pulls in this step has no use for a gradient (Algorithm 1 takes one branch or the
     // other), so nothing is transferred for it.

@@ -244,8 +244,14 @@ def test_step_host_transfers_no_gradient_for_workers_that_pull_and_splits_the_st
         gpu.set_grads(marker)                                     # what the device buffers held before the call
         g = _grads(cfg, P, t)
         hg.copy_(torch.from_numpy(g))
-        gpu.lib.step_host(gp, cfg.lr, cfg.eta, None, 0, gpu.stream)
+        # pulling workers need no gradient at all: their host pointers may be NULL
+        import paper_2504_18454_b200 as PL
+        pulls = [PL.decision(cfg.decision_seed, t, k, cfg.p) for k in range(cfg.K)]
+        gp_t = gpu.lib.make_ptr_array([0 if pulls[k] else hg.data_ptr() + (k * P + int(starts[j])) * 4
+                                       for k in range(cfg.K) for j in range(len(numel))])
+        gpu.lib.step_host(gp_t if t % 2 else gp, cfg.lr, cfg.eta, None, 0, gpu.stream)
         orc.step(g, cfg.lr, cfg.eta)
+        assert pulls == [int(v) for v in orc.last_b]
         on_device = gpu._read("grad")
         for k in range(cfg.K):
             want = marker[k] if orc.last_b[k] else g[k]           # pulled: untouched; gradient step: copied
