@@ -303,7 +303,7 @@ int palsgd_get_launch_count(palsgd_ctx* ctx, uint64_t* n_launches);
  * kernel: 0 = worker index fastest (default), 1 = chunk index fastest.
  * OUTER_SUB_ELEMS: elements per work item of the outer kernel (a slice of a chunk),
  * a multiple of 1024; default 1024 (4096 for K < 8).
- * DDP_SUB_ELEMS: the same for the DDP warm-up kernel; default 2048 (4096 in BF16_MASTER mode).
+ * DDP_SUB_ELEMS: the same for the DDP warm-up kernel; default 1024 (4096 in BF16_MASTER mode).
  * DDP_VARIANT: how the DDP warm-up kernel writes its result to the K slots: 1 = 128-bit stores
  * by every thread, 2 = staged in shared memory and fanned out by bulk asynchronous stores;
  * 0 = the library's default (2).

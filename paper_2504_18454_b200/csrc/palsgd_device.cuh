@@ -13,7 +13,8 @@ constexpr uint32_t kChunkElems  = 8192;    // default elements per chunk-table e
 constexpr uint32_t kStageElems  = 4096;    // stage size of the shared-memory-ring kernels
 constexpr uint32_t kOuterSubElems = 1024;  // default work item of the outer kernel for K >= 8: a slice of a
                                            // chunk (small: K+2 streams per element need many CTAs in flight)
-constexpr uint32_t kDdpSubElems = 2048;    // default work item of the DDP warm-up kernel (measured)
+constexpr uint32_t kDdpSubElems = 1024;    // default work item of the DDP warm-up kernel in fp32 mode (measured
+                                           // with the persistent grid; 4096 in bf16 mode)
 constexpr uint32_t kSegVecFlag  = 0x80000000u;   // Chunk::seg bit: 16-byte vector path allowed
 
 // One work unit of the multi-tensor launch: `len` consecutive elements of
