@@ -108,7 +108,7 @@ typedef struct palsgd_buffers {
 
 /*
  * Create a context (Algorithm 1, initialisation).  Validates everything before
- * touching the GPU.  Then, on `stream`: m, v, outer_mom <- 0; global[i] <-
+ * touching the GPU.  Then, on `stream`: m, v, outer_mom (and outer_v) <- 0; global[i] <-
  * (x_0[i] + x_1[i] + ... + x_{K-1}[i]) / K, summed in that order (Sec. 2.2; the
  * paper starts all workers from one x^(0), for which this is x^(0)); in
  * BF16_MASTER mode param <- RNE_bf16(master).  Counters t, s_k, n_outer <- 0.
@@ -120,7 +120,8 @@ int palsgd_init(palsgd_ctx** out, const palsgd_config* cfg, size_t n_tensors,
                 const uint64_t* numel, const palsgd_buffers* bufs, void* stream);
 
 /*
- * One pass of Algorithm 1's inner loop body for all K workers, ONE kernel launch.
+ * One pass of Algorithm 1's inner loop body for all K workers, ONE kernel launch (one
+ * more, ahead of it, while gradient clipping is on: see palsgd_set_grad_clip).
  * For worker k the kernel draws b_k^(t) ("b ~ U[0,1]; b <= p"): the first word r of
  * Philox4x32-10 with key (seed_lo, seed_hi) and counter (t_lo, t_hi, k, 0);
  * b = (r < floor(p * 2^32)).  One draw per (worker, step) for the whole model.
