@@ -234,7 +234,8 @@ def workload_config(cfg, args) -> dict:
             "p": cfg.p, "eta": cfg.eta, "lr": cfg.lr,
             "inner": "adamw" if cfg.inner == 0 else "sgdm",
             "precision": "bf16 params+grads, fp32 master/moments" if cfg.precision == 1 else "fp32",
-            "parallelism": f"replicas x{args.gpus}" if args.gpus > 1 else "single GPU",
+            "parallelism": (f"parameter-axis shards x{args.gpus}" if getattr(args, "shard", False)
+                            else f"replicas x{args.gpus}") if args.gpus > 1 else "single GPU",
             "l2": "state far larger than L2 (no flush needed)"
                   if cfg.K * cfg.P * 16 > 4 * 126e6 else "L2-affected: state comparable to the 126 MB L2"}
 
@@ -286,8 +287,15 @@ def run_ours(args, cfg):
     # ---- buffers: seeded synthetic values, resident in HBM
     K, Pn = cfg.K, cfg.P
     numel = [t.numel for t in cfg.tensors]
+    P_job = Pn * world                      # elements per worker over the whole job (replicas: one model per rank)
+    if args.shard:
+        # strong scaling: ONE model, every rank owns a slice of the parameter axis of all K slots;
+        # the path is elementwise and the decisions depend on (seed, t, k) only, so no exchange is needed
+        from paper_2504_18454_b200.shard import shard_numel
+        numel = shard_numel(numel, rank, world)
+        P_job, Pn = Pn, int(sum(numel))
     arena = ReplicaArena(numel, K, precision=cfg.precision, inner=cfg.inner, device=dev)
-    x_init = torch.from_numpy(W.init_params_host(cfg.tensors, cfg.param_seed + rank, cfg.init_std)).to(dev)
+    x_init = torch.from_numpy(W.init_params_host(cfg.tensors, cfg.param_seed + rank, cfg.init_std))[:Pn].to(dev)
     arena.model.copy_(x_init[None].expand(K, Pn))
     gen = torch.Generator(device=dev)
     gen.manual_seed(cfg.grad_seed + rank)
@@ -423,13 +431,13 @@ def run_ours(args, cfg):
         e2e["ms"] = ms_e2e_max
     if rank == 0:
         peak, peak_src = measured_peak_gbs()
-        value = whole_job_value(world, K, Pn, args.steps, ms_total)
+        value = whole_job_value(1, K, P_job, args.steps, ms_total)
         inner_gbs = inner_bytes / (inner_ms * 1e-3) / 1e9 if inner_ms else None
         outer_gbs = outer_bytes / (outer_ms * 1e-3) / 1e9 if outer_ms else None
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_total / args.steps,
-            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "higher_is_better": True, "scaling": "strong" if args.shard else "weak", "vs_baseline": None,
             "dtype": "f32",
             "data": "synthetic", "config": workload_config(cfg, args),
             "roofline": {"bound": "hbm", "kernel": "palsgd_inner_kernel", "achieved": inner_gbs,
@@ -457,7 +465,7 @@ def run_ours(args, cfg):
                               "note": "timed outside the step loop; not part of value"} if ddp else None),
             "graph_cycle": graph_cycle,
             "cpu_baseline": cpu_baseline,
-            "e2e": ({"value": world * K * Pn * e2e["steps"] / (e2e["ms"] * 1e-3), "unit": UNIT,
+            "e2e": ({"value": K * P_job * e2e["steps"] / (e2e["ms"] * 1e-3), "unit": UNIT,
                      "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
                      "steps": e2e["steps"], "outer_syncs": e2e["syncs"]} if e2e else None),
             "gpu_launches": launches,
@@ -480,6 +488,9 @@ def main():
     ap.add_argument("--inner-variant", type=int, default=0, help="palsgd_set_tuning(INNER_VARIANT); 0 = default")
     ap.add_argument("--grad-clip", type=float, default=0.0,
                     help="global-norm clip threshold (adds the norm pass to every step); 0 = off, the benchmark default")
+    ap.add_argument("--shard", action="store_true",
+                    help="N > 1: one model sharded over the ranks along the parameter axis (strong scaling, no "
+                         "exchange) instead of one replica of the workload per rank")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="skip the separate timing of the graph-captured cycle")
