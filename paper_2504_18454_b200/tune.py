@@ -125,6 +125,22 @@ def _child(args) -> None:
                        for i in range(steps) for k in range(cfg.K)) * cfg.P
         return byts / (clipped - base) / 1e6, (clipped - base) / steps, base / steps
 
+    def time_pull(reps=8):
+        mask = (1 << cfg.K) - 1
+        for _ in range(2):
+            ctx.pseudo_sync(mask, 0.1, stream)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            ctx.pseudo_sync(mask, 0.1, stream)
+        e1.record()
+        torch.cuda.synchronize()
+        per = 14 if cfg.precision == 1 else 12
+        return per * cfg.K * cfg.P / (e0.elapsed_time(e1) / reps) / 1e6
+
+    r = sorted(time_pull() for _ in range(3))
+    print(f"{cfg.name} chunk={chunk} forced pull of all workers: {r[1]:.0f} GB/s (runs {r[0]:.0f}..{r[2]:.0f}; "
+          f"x_g shared through L2, so the floor is below the 12/14 B per element assumed)", flush=True)
     for v in args.variants:
         ctx.set_tuning(P.TUNE_INNER_VARIANT, v)
         r = sorted(time_inner(args.steps) for _ in range(3))
