@@ -13,3 +13,5 @@ def test_oracle_output_unchanged_since_golden_was_written():
     spec.loader.exec_module(mod)
     with open(os.path.join(HERE, "golden", "oracle_tiny_run.txt")) as f:
         assert mod.render() == f.read()
+    with open(os.path.join(HERE, "golden", "oracle_widened_run.txt")) as f:      # warm-up, clipping, AdamW outer
+        assert mod.render_widened() == f.read()
