@@ -114,6 +114,22 @@ def whole_job_value(world: int, K: int, P: int, steps: int, ms_total: float) -> 
     return world * K * P * steps / (ms_total * 1e-3)
 
 
+def rank_share(numel, rank: int, world: int, shard: bool):
+    """What one rank of the job holds.  Replicas (default): the whole tensor list, a model of its own
+    (seed offset = rank), so the job updates world * P elements per worker and step (weak scaling).
+    Shards: its slice [lo, hi) of the parameter axis of ONE model (seed offset 0), so the job updates P
+    elements per worker and step however many ranks there are (strong scaling).
+    Returns (numel of the rank's tensor list, lo, hi, seed offset, elements per worker of the whole job)."""
+    P = int(sum(numel))
+    if not shard:
+        return [int(n) for n in numel], 0, P, rank, P * world
+    from paper_2504_18454_b200.shard import shard_numel, shard_span
+    lo, hi = shard_span(numel, rank, world)
+    mine = shard_numel(numel, rank, world)
+    assert hi - lo == sum(mine)
+    return mine, lo, hi, 0, P
+
+
 class ClockSampler:
     """nvidia-smi clock / throttle sampling while the timed region runs."""
 
@@ -209,8 +225,7 @@ def run_reference(args, cfg):
     if rank != 0:
         return
     P_sample = min(cfg.P, 1 << 21)
-    H = max(2, min(cfg.H, args.steps))
-    t_all = []
+    H = cfg.H                                   # the workload's own interval, as printed in `config`
     for _ in range(max(args.warmup, 0)):
         time_oracle(cfg, 1, P_sample, H)
     value, dt, cores, n_outer = time_oracle(cfg, args.steps, P_sample, H)
@@ -220,7 +235,7 @@ def run_reference(args, cfg):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f32",
+        "dtype": dtype_of(cfg),
         "data": "synthetic", "config": workload_config(cfg, args),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -229,8 +244,33 @@ def run_reference(args, cfg):
     print(json.dumps(line), flush=True)
 
 
+def dtype_of(cfg) -> str:
+    """The arithmetic type of the path (every element operation is binary32), with the storage types
+    of the mixed-precision workloads spelled out."""
+    return "f32" if cfg.precision == 0 else "f32 arithmetic; bf16 params+grads, f32 master/moments"
+
+
+def roofline_entry(kernel: str, kind: str, cfg, peak: float, peak_src: str, ms_sum: float, bytes_sum: float,
+                   n: int, units_per_launch: int = 0, **extra) -> dict:
+    """One roofline object: achieved = algorithmic bytes / CUDA-event time of the kernel's launches."""
+    gbs = bytes_sum / (ms_sum * 1e-3) / 1e9 if ms_sum else None
+    d = {"bound": "hbm", "kernel": kernel, "achieved": gbs, "peak": peak, "unit": "GB/s",
+         "frac": gbs / peak if gbs else None,
+         "traffic": ncu_traffic(kind, cfg.precision, bytes_sum / n if n else None),
+         "peak_source": peak_src,
+         "frac_of_measured_copy": gbs / peak if gbs else None,
+         "frac_of_nominal_peak": gbs / 8000.0 if gbs else None, "nominal_peak": 8000.0,
+         "launches": n, "avg_ms": ms_sum / n if n else None,
+         "alg_bytes_per_launch": bytes_sum / n if n else None}
+    if units_per_launch and ms_sum:
+        d["params_per_s"] = units_per_launch * n / (ms_sum * 1e-3)
+    d.update(extra)
+    return d
+
+
 def workload_config(cfg, args) -> dict:
     return {"workload": cfg.name, "K": cfg.K, "P": cfg.P, "n_tensors": len(cfg.tensors), "H": cfg.H,
+            "layout": getattr(args, "layout", "arena"),
             "p": cfg.p, "eta": cfg.eta, "lr": cfg.lr,
             "inner": "adamw" if cfg.inner == 0 else "sgdm",
             "precision": "bf16 params+grads, fp32 master/moments" if cfg.precision == 1 else "fp32",
@@ -285,29 +325,28 @@ def run_ours(args, cfg):
                         "single_thread_sample": f"first {P_1} elements per worker, {n_1} steps, {dt1:.1f} s"}
 
     # ---- buffers: seeded synthetic values, resident in HBM
-    K, Pn = cfg.K, cfg.P
-    numel = [t.numel for t in cfg.tensors]
-    P_job = Pn * world                      # elements per worker over the whole job (replicas: one model per rank)
-    if args.shard:
-        # strong scaling: ONE model, every rank owns a slice of the parameter axis of all K slots;
-        # the path is elementwise and the decisions depend on (seed, t, k) only, so no exchange is needed
-        from paper_2504_18454_b200.shard import shard_numel
-        numel = shard_numel(numel, rank, world)
-        P_job, Pn = Pn, int(sum(numel))
-    arena = ReplicaArena(numel, K, precision=cfg.precision, inner=cfg.inner, device=dev)
-    x_init = torch.from_numpy(W.init_params_host(cfg.tensors, cfg.param_seed + rank, cfg.init_std))[:Pn].to(dev)
-    arena.model.copy_(x_init[None].expand(K, Pn))
+    K = cfg.K
+    # shards: every rank owns a slice of the parameter axis of all K slots of ONE model; the path is
+    # elementwise and the decisions depend on (seed, t, k) only, so no exchange is needed
+    numel, lo, hi, seed_off, P_job = rank_share([t.numel for t in cfg.tensors], rank, world, args.shard)
+    Pn = hi - lo
+    arena = ReplicaArena(numel, K, precision=cfg.precision, inner=cfg.inner, device=dev, layout=args.layout)
+    x_full = W.init_params_host(cfg.tensors, cfg.param_seed + seed_off, cfg.init_std)
+    x_init = torch.from_numpy(x_full[lo:lo + Pn]).to(dev)
+    del x_full
+    for k in range(K):
+        arena.write_flat(arena.model_name, k, x_init)
     gen = torch.Generator(device=dev)
     gen.manual_seed(cfg.grad_seed + rank)
     for k in range(K):
-        arena.rows("grad")[k].copy_(
-            torch.randn(Pn, generator=gen, device=dev, dtype=torch.float32).mul_(cfg.grad_std))
+        arena.write_flat("grad", k, torch.randn(Pn, generator=gen, device=dev, dtype=torch.float32).mul_(cfg.grad_std))
     del x_init
     stream = torch.cuda.current_stream(dev).cuda_stream
     ctx = arena.make_context(
         stream=stream, H=cfg.H, p=cfg.p, beta1=cfg.beta1, beta2=cfg.beta2, eps=cfg.eps,
         weight_decay=cfg.weight_decay, momentum=cfg.momentum, outer_lr=cfg.outer_lr,
         outer_momentum=cfg.outer_momentum, outer_nesterov=cfg.outer_nesterov, seed=cfg.decision_seed)
+    layout_info = ctx.get_layout()
 
     if args.inner_variant:
         ctx.set_tuning(P.TUNE_INNER_VARIANT, args.inner_variant)
@@ -346,7 +385,6 @@ def run_ours(args, cfg):
     barrier()
     ms_total = e_start.elapsed_time(e_end)
     launches = ctx.get_launch_count() - launches0
-    clocks = sampler.stop() if rank == 0 else None
     events.append(("end", t_host, e_end))
 
     # per-kernel durations (event to next event on the same stream) and algorithmic bytes
@@ -360,13 +398,34 @@ def run_ours(args, cfg):
             inner_ms += d; inner_bytes += b; n_inner += 1
         else:
             outer_ms += d; outer_bytes += outer_bytes_per_param(cfg) * Pn; n_outer += 1
+    in_loop_outer = n_outer
+
+    # ---- the outer-sync kernel on its own (the metric's "per outer_sync" half), whatever --steps is:
+    # launches behind slots that two inner steps have let diverge again, one CUDA-event pair each,
+    # under the same load (and clocks) as the step loop, which continues around them
+    outer_alone = []
+    if not args.no_outer:
+        for i in range(args.outer_launches + 1):
+            for _ in range(2):
+                ctx.inner_step(cfg.lr, cfg.eta, stream); t_host += 1
+            e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+            e0.record()
+            ctx.outer_sync(stream)
+            e1.record()
+            if i > 0:                                    # the first one is a warm-up
+                outer_alone.append((e0, e1))
+        torch.cuda.synchronize(dev)
+        for e0, e1 in outer_alone:
+            outer_ms += e0.elapsed_time(e1); outer_bytes += outer_bytes_per_param(cfg) * Pn; n_outer += 1
+    clocks = sampler.stop() if rank == 0 else None
 
     # ---- end to end: gradients from pinned host memory, results back to the host, every step
     e2e = None
     if not args.no_e2e:
         gdt = torch.bfloat16 if cfg.precision == 1 else torch.float32
         h_grad = torch.empty((K, Pn), dtype=gdt).pin_memory()
-        h_grad.copy_(arena.rows("grad"))
+        for k in range(K):
+            h_grad[k].copy_(arena.read_flat("grad", k))
         h_glob = torch.empty(Pn, dtype=torch.float32).pin_memory()
         h_dec = torch.zeros(K, dtype=torch.uint8).pin_memory()
         es = h_grad.element_size()
@@ -422,8 +481,8 @@ def run_ours(args, cfg):
             ctx.ddp_step(cfg.lr, stream)
             evs[i + 1].record()
         torch.cuda.synchronize(dev)
-        ddp_ms = sum(evs[i].elapsed_time(evs[i + 1]) for i in range(8)) / 8
-        ddp = {"avg_ms": ddp_ms, "alg_bytes_per_launch": ddp_bytes_per_param(cfg) * Pn, "launches": 8}
+        ddp_ms = sum(evs[i].elapsed_time(evs[i + 1]) for i in range(8))
+        ddp = {"ms": ddp_ms, "bytes": 8 * ddp_bytes_per_param(cfg) * Pn, "launches": 8}
 
     # ---- max over ranks
     ms_total, ms_e2e_max = max_over_ranks([ms_total, e2e["ms"] if e2e else 0.0], world, dev)
@@ -432,37 +491,31 @@ def run_ours(args, cfg):
     if rank == 0:
         peak, peak_src = measured_peak_gbs()
         value = whole_job_value(1, K, P_job, args.steps, ms_total)
-        inner_gbs = inner_bytes / (inner_ms * 1e-3) / 1e9 if inner_ms else None
-        outer_gbs = outer_bytes / (outer_ms * 1e-3) / 1e9 if outer_ms else None
+        r_inner = roofline_entry("palsgd_inner_kernel", "inner", cfg, peak, peak_src, inner_ms, inner_bytes, n_inner)
+        r_outer = roofline_entry("palsgd_outer_kernel", "outer", cfg, peak, peak_src, outer_ms, outer_bytes, n_outer,
+                                 units_per_launch=Pn, launches_inside_step_loop=in_loop_outer,
+                                 launches_timed_alone=n_outer - in_loop_outer,
+                                 note="launches inside the step loop plus launches timed on their own right "
+                                      "after it, each behind slots that inner steps have let diverge")
+        cycle = None
+        if r_inner["avg_ms"] and r_outer["avg_ms"]:
+            # average cost per step of a whole synchronisation cycle: H inner launches + one outer sync
+            cyc_ms = (cfg.H * r_inner["avg_ms"] + r_outer["avg_ms"]) / cfg.H
+            cycle = {"H": cfg.H, "ms_per_step": cyc_ms, "value": K * Pn / (cyc_ms * 1e-3), "unit": UNIT,
+                     "outer_share": r_outer["avg_ms"] / (cfg.H * cyc_ms),
+                     "note": "(H * inner avg + outer avg) / H from the per-kernel CUDA-event times above"}
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_total / args.steps,
             "higher_is_better": True, "scaling": "strong" if args.shard else "weak", "vs_baseline": None,
-            "dtype": "f32",
-            "data": "synthetic", "config": workload_config(cfg, args),
-            "roofline": {"bound": "hbm", "kernel": "palsgd_inner_kernel", "achieved": inner_gbs,
-                         "peak": peak, "unit": "GB/s", "frac": inner_gbs / peak if inner_gbs else None,
-                         "traffic": ncu_traffic("inner", cfg.precision, inner_bytes / n_inner if n_inner else None),
-                         "peak_source": peak_src, "frac_of_8000_nominal":
-                         inner_gbs / 8000.0 if inner_gbs else None,
-                         "launches": n_inner, "avg_ms": inner_ms / n_inner if n_inner else None,
-                         "alg_bytes_per_launch": inner_bytes / n_inner if n_inner else None},
-            "roofline_outer": {"bound": "hbm", "kernel": "palsgd_outer_kernel", "achieved": outer_gbs,
-                               "peak": peak, "unit": "GB/s", "frac": outer_gbs / peak if outer_gbs else None,
-                               "traffic": ncu_traffic("outer", cfg.precision, outer_bytes / n_outer if n_outer else None),
-                               "frac_of_8000_nominal": outer_gbs / 8000.0 if outer_gbs else None,
-                               "launches": n_outer, "avg_ms": outer_ms / n_outer if n_outer else None,
-                               "alg_bytes_per_launch": outer_bytes / n_outer if n_outer else None,
-                               "params_per_s": Pn * n_outer / (outer_ms * 1e-3) if outer_ms else None},
-            "roofline_ddp": ({"bound": "hbm", "kernel": "palsgd_ddp_kernel",
-                              "achieved": ddp["alg_bytes_per_launch"] / (ddp["avg_ms"] * 1e-3) / 1e9,
-                              "peak": peak, "unit": "GB/s",
-                              "frac": ddp["alg_bytes_per_launch"] / (ddp["avg_ms"] * 1e-3) / 1e9 / peak,
-                              "traffic": ncu_traffic("ddp", cfg.precision, ddp["alg_bytes_per_launch"]),
-                              "launches": ddp["launches"], "avg_ms": ddp["avg_ms"],
-                              "alg_bytes_per_launch": ddp["alg_bytes_per_launch"],
-                              "params_per_s": Pn / (ddp["avg_ms"] * 1e-3),
-                              "note": "timed outside the step loop; not part of value"} if ddp else None),
+            "dtype": dtype_of(cfg),
+            "data": "synthetic", "config": dict(workload_config(cfg, args), **layout_info),
+            "roofline": r_inner,
+            "roofline_outer": r_outer,
+            "cycle": cycle,
+            "roofline_ddp": (roofline_entry("palsgd_ddp_kernel", "ddp", cfg, peak, peak_src, ddp["ms"], ddp["bytes"],
+                                            ddp["launches"], units_per_launch=Pn,
+                                            note="timed outside the step loop; not part of value") if ddp else None),
             "graph_cycle": graph_cycle,
             "cpu_baseline": cpu_baseline,
             "e2e": ({"value": K * P_job * e2e["steps"] / (e2e["ms"] * 1e-3), "unit": UNIT,
@@ -491,6 +544,12 @@ def main():
     ap.add_argument("--shard", action="store_true",
                     help="N > 1: one model sharded over the ranks along the parameter axis (strong scaling, no "
                          "exchange) instead of one replica of the workload per rank")
+    ap.add_argument("--layout", choices=["arena", "separate", "misaligned"], default="arena",
+                    help="device layout of the tensor list: packed (K, P) arenas (default), one allocation per "
+                         "(worker, tensor, buffer kind), or packed and shifted off 16-byte alignment")
+    ap.add_argument("--outer-launches", type=int, default=8,
+                    help="outer-sync launches timed on their own after the step loop")
+    ap.add_argument("--no-outer", action="store_true", help="skip the separate timing of the outer-sync kernel")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="skip the separate timing of the graph-captured cycle")

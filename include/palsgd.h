@@ -56,7 +56,7 @@ typedef enum palsgd_status {
     PALSGD_ESTATE       = -4,   /* call not valid in this state (e.g. undefined coefficient)         */
     PALSGD_ENOMEM       = -5,   /* host or device allocation failed                                  */
     PALSGD_EUNSUPPORTED = -6,   /* combination not built                                             */
-    PALSGD_ETIMEOUT     = -7,   /* a bounded wait inside a kernel expired (reported by get_counters)  */
+    /* -7 is not used */
     PALSGD_ETOOBIG      = -8    /* tensor list needs more than the fixed scratch of a no-allocation call */
 } palsgd_status;
 
@@ -122,7 +122,7 @@ int palsgd_init(palsgd_ctx** out, const palsgd_config* cfg, size_t n_tensors,
 /*
  * One pass of Algorithm 1's inner loop body for all K workers, ONE kernel launch (one
  * more, ahead of it, while gradient clipping is on: see palsgd_set_grad_clip).
- * For worker k the kernel draws b_k^(t) ("b ~ U[0,1]; b <= p"): the first word r of
+ * For worker k the kernel draws b_k^(t), Algorithm 1's uniform variate compared with p: the first word r of
  * Philox4x32-10 with key (seed_lo, seed_hi) and counter (t_lo, t_hi, k, 0);
  * b = (r < floor(p * 2^32)).  One draw per (worker, step) for the whole model.
  *   b = 1, Eq. (2):  d = x - x_g;  x = x - beta * d,   beta = fl32(alpha_t*eta_t/p).
@@ -185,6 +185,35 @@ int palsgd_pseudo_sync(palsgd_ctx* ctx, uint64_t worker_mask, double beta, void*
  */
 int palsgd_outer_sync(palsgd_ctx* ctx, void* stream);
 
+/*
+ * The outer synchronisation when the K workers of Algorithm 1 are spread over several GPUs
+ * (the deployment the paper itself runs: Algorithm 1's All-Reduce of the outer gradient across
+ * workers, an average by Sec. 2.2).  Each GPU holds a context over its K_local workers; the
+ * exchange is the caller's collective (e.g. one NCCL all-reduce(sum)), the library supplies the
+ * two kernels around it:
+ *   1. palsgd_outer_partial:  exchange[i] = x_0[i] + x_1[i] + ... + x_{K_local-1}[i]  (that order)
+ *   2. the caller sums the exchange buffers of all GPUs element by element (all-reduce, sum)
+ *   3. palsgd_outer_finish:   xbar = exchange[i] / K_total;  then exactly palsgd_outer_sync's
+ *      Delta, OuterOPT update of x_g (Eq. (3), Eq. (4)) and the restart of the K_local slots.
+ * With one GPU (K_total = K_local, step 2 empty) the result is bit-identical to
+ * palsgd_outer_sync.  With G GPUs the sum over k is grouped by GPU, and the order in which step
+ * 2 adds the G partial sums is the collective's; the result then differs from the single-GPU one
+ * by rounding only (for G = 2 it is one commutative addition, hence unique).  Every GPU must
+ * call with the same outer learning rate and K_total; all end with the same x_g and u.
+ * The exchange buffer is device memory of palsgd_exchange_numel() floats (the total element
+ * count), 16-byte aligned, caller-owned: the tensor list packed back to back, tensor j at the
+ * sum of the element counts before it -- the same on every GPU whatever its memory layout.
+ * palsgd_outer_finish counts as the outer sync: n_outer += 1.
+ * palsgd_set_worker_offset(k0) makes the local workers draw their decisions as workers
+ * k0 .. k0+K_local-1 of the job (Algorithm 1's worker index); default 0.
+ * Errors: EINVAL (NULL, K_total < K_local, k0 + K_local > 2^32); EALIGN; EUNSUPPORTED (an
+ * OUTER_SUB_ELEMS value whose stage does not fit in shared memory); ECUDA.
+ */
+int palsgd_exchange_numel(palsgd_ctx* ctx, uint64_t* n_floats);
+int palsgd_set_worker_offset(palsgd_ctx* ctx, uint32_t k0);
+int palsgd_outer_partial(palsgd_ctx* ctx, float* exchange, void* stream);
+int palsgd_outer_finish(palsgd_ctx* ctx, const float* exchange, uint32_t K_total, void* stream);
+
 /* The outer learning rate of the following outer syncs (it may follow a schedule, e.g. the
  * warm-up + cosine annealing of Appendix B: see palsgd_schedule_value).  Errors: EINVAL. */
 int palsgd_set_outer_lr(palsgd_ctx* ctx, double outer_lr);
@@ -193,7 +222,7 @@ int palsgd_set_outer_lr(palsgd_ctx* ctx, double outer_lr);
  * Pure host function: the value at step t of a schedule with a linear warm-up over
  * `warmup` steps from base*start_factor to base, followed by a constant
  * (PALSGD_SCHED_WARMUP_CONSTANT) or by cosine annealing down to min_value at step `total`
- * (PALSGD_SCHED_WARMUP_COSINE; Appendix B: "a warm-up period ... followed by cosine annealing"):
+ * (PALSGD_SCHED_WARMUP_COSINE; the outer learning-rate schedule of Appendix B):
  *   t <  warmup: base * (start_factor + (1 - start_factor) * t / warmup)
  *   t >= warmup: base, or min_value + (base - min_value) * (1 + cos(pi*tau/(total - warmup))) / 2
  *                with tau = min(t, total) - warmup.
@@ -255,8 +284,7 @@ int palsgd_step_host(palsgd_ctx* ctx, const void* const* h_grad, double lr_t, do
  * Read the counters (SYNCHRONISES the stream): t = completed steps, s_k[K] =
  * gradient steps taken by worker k, n_outer = outer syncs, last_b[K] = decisions
  * of the latest inner step.  Any output pointer may be NULL.
- * Errors: ETIMEOUT if a kernel recorded an expired wait; ESTATE if the device-side
- * t disagrees with the host mirror; ECUDA.
+ * Errors: ESTATE if the device-side t disagrees with the host mirror; ECUDA.
  */
 int palsgd_get_counters(palsgd_ctx* ctx, uint64_t* t, uint64_t* s_k, uint64_t* n_outer,
                         uint8_t* last_b, void* stream);
@@ -267,8 +295,8 @@ int palsgd_set_counters(palsgd_ctx* ctx, uint64_t t, const uint64_t* s_k, uint64
                         void* stream);
 
 /*
- * Global-norm gradient clipping (Appendix B trains GPT-Neo "with gradient clipping
- * enabled" and gives no threshold, so it is a parameter here).  max_norm > 0 turns it
+ * Global-norm gradient clipping (Appendix B: the GPT-Neo runs clip their gradients; no
+ * threshold is given, so it is a parameter here).  max_norm > 0 turns it
  * on for the following palsgd_inner_step / palsgd_step / palsgd_ddp_step calls,
  * 0 turns it off (the default).  Convention of the software the paper ran
  * (clip_grad_norm_), per worker k that takes a gradient step:
@@ -291,38 +319,34 @@ int palsgd_get_grad_norms(palsgd_ctx* ctx, double* sumsq, float* clip, void* str
 /* Number of kernels this context has launched so far (host-side count). */
 int palsgd_get_launch_count(palsgd_ctx* ctx, uint64_t* n_launches);
 
+/* What palsgd_init made of the tensor list (the multi-tensor launch metadata): the number of
+ * segments (maximal runs of tensors that are adjacent in memory in every buffer), of chunk-table
+ * entries (pieces of a segment of at most *chunk_elems elements; one work item of the inner kernel
+ * per worker each) and the chunk size.  Any output pointer may be NULL.  Errors: EINVAL. */
+int palsgd_get_layout(palsgd_ctx* ctx, uint64_t* n_segments, uint64_t* n_chunks, uint32_t* chunk_elems);
+
 /* Launch-shape knobs (advanced; results never depend on them).
  * *_GRID_CAP: the largest grid a launch may use, CTAs looping over work items
  * beyond it; 0 (default) = one CTA per work item.
- * INNER_VARIANT: which form of the fused inner kernel runs: 0 = the library's default (the measured
- * best launch shape as a persistent grid that draws its work items from a queue in device memory);
- * 18 = the same shape with one CTA per work item; 1..9, 13..15 = other register-path shapes (loads in
- * flight per thread x CTAs per SM), one CTA per item; 10 / 11 / 12 = the persistent shared-memory-ring
- * form with 512 / 256 / 1024 consumer threads; unknown = default.
- * PIPE_STAGES: ring depth of the persistent form; 0 = as many as fit.
- * CHUNK_MAJOR: order of the (chunk, worker) work items of the register-path inner
- * kernel: 0 = worker index fastest (default), 1 = chunk index fastest.
- * OUTER_SUB_ELEMS: elements per work item of the outer kernel (a slice of a chunk),
- * a multiple of 1024; default 1024 (4096 for K < 8).
- * DDP_SUB_ELEMS: the same for the DDP warm-up kernel; default 1024 (4096 in BF16_MASTER mode).
+ * INNER_VARIANT: 0 = the fused inner kernel as a persistent grid that draws its work items from a
+ * queue in device memory (default); 18 = the same kernel with one CTA per work item.
+ * OUTER_SUB_ELEMS: elements per work item of the outer kernel, a multiple of 1024; default 1024
+ * (4096 for K < 8).  DDP_SUB_ELEMS: the same for the DDP warm-up kernel.  Setting either rebuilds
+ * a device table: the call synchronises the device and must not be made during stream capture.
  * DDP_VARIANT: how the DDP warm-up kernel writes its result to the K slots: 1 = 128-bit stores
  * by every thread, 2 = staged in shared memory and fanned out by bulk asynchronous stores;
  * 0 = the library's default (2).
  * OUTER_VARIANT: the same choice for the outer-sync kernel.
  * OUTER_DYNAMIC: outer-sync and DDP kernels as a persistent grid of that many CTAs per SM that
  * draws its work items from a queue; 0 = one CTA per work item.  Until this knob is set the
- * library uses its defaults (outer sync: one CTA per item; DDP step: 4 CTAs per SM).
- * (Environment variable PALSGD_CHUNK_ELEMS, read by palsgd_init: elements per chunk
- * = per work item of the inner kernel, a multiple of 1024; default 4096 for fp32 AdamW,
- * 8192 otherwise.) */
+ * library uses its defaults. */
 enum { PALSGD_TUNE_INNER_GRID_CAP = 0, PALSGD_TUNE_OUTER_GRID_CAP = 1, PALSGD_TUNE_INNER_VARIANT = 2,
-       PALSGD_TUNE_PIPE_STAGES = 3, PALSGD_TUNE_CHUNK_MAJOR = 4, PALSGD_TUNE_OUTER_SUB_ELEMS = 5,
-       PALSGD_TUNE_DDP_SUB_ELEMS = 6, PALSGD_TUNE_DDP_VARIANT = 7,
+       PALSGD_TUNE_OUTER_SUB_ELEMS = 5, PALSGD_TUNE_DDP_SUB_ELEMS = 6, PALSGD_TUNE_DDP_VARIANT = 7,
        PALSGD_TUNE_OUTER_VARIANT = 8, PALSGD_TUNE_OUTER_DYNAMIC = 9 };
 int palsgd_set_tuning(palsgd_ctx* ctx, int knob, int64_t value);
 
 /* The branch draw as a pure host function: 1 = pseudo-sync, 0 = gradient step;
- * negative status on bad arguments (p outside [0,1], k >= 64). */
+ * negative status on bad arguments (p outside [0,1]).  k is the worker's index in the job. */
 int palsgd_decision(uint64_t seed, uint64_t t, uint32_t k, double p);
 
 /* Text for a status; the CUDA error string of the latest ECUDA on ctx (or ""). */
@@ -349,9 +373,12 @@ const char* palsgd_last_cuda_error(palsgd_ctx* ctx);
  * master = fp32 local models (averaged and rewritten), param = bf16 working
  * copies (rewritten as RNE of the new global model).  numel[j] = 0 is allowed.
  * The call rebuilds the tables, copies them into the array on `stream`, and
- * launches one kernel on `stream`; it does not synchronise.  It calls neither
- * cudaMalloc nor cudaFree nor any other allocating routine, on the device or on
- * the host.
+ * launches one kernel on `stream`.  It calls neither cudaMalloc nor cudaFree nor
+ * any other allocating routine, on the device or on the host.  The tables come
+ * from ordinary (pageable) host memory inside the library, so the copy makes
+ * the HOST wait until the work enqueued on `stream` before this call has
+ * finished; the kernel itself then runs asynchronously, and work on other
+ * streams is not affected.
  *
  * Limit: the tables need 16 bytes per started block of 8192 elements of every
  * tensor, plus 8 bytes per (worker, non-empty tensor) pointer (twice that in
@@ -369,8 +396,14 @@ const char* palsgd_last_cuda_error(palsgd_ctx* ctx);
  *
  * First call on each device: looks up the array's device address (a runtime
  * call that is made once per device and cached, with that device current).
- * Make this first call outside any stream capture.
- * Errors: EINVAL, EALIGN, ETOOBIG before any CUDA call; ECUDA.
+ *
+ * Never under stream capture, first call or later: the table copy would be
+ * recorded as a node that re-reads the library's host buffer, and the kernel
+ * node would keep this call's table sizes, at every replay, after later calls
+ * have put other tables there.  A call on a capturing stream returns
+ * PALSGD_ESTATE and enqueues nothing.
+ * Errors: EINVAL, EALIGN, ETOOBIG before any CUDA call; ESTATE (capturing
+ * stream); ECUDA.
  */
 #define PALSGD_NOALLOC_SCRATCH_BYTES (1u << 20)
 int palsgd_outer_sync_noalloc(uint32_t K, int32_t precision, size_t n_tensors,

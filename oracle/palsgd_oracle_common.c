@@ -190,8 +190,7 @@ double palsgd_oracle_clip_coef(double sumsq, double max_norm)
 
 /* Value at step t of a schedule with a linear warm-up followed by a constant
  * (kind 0) or by cosine annealing (kind 1), the form the paper's experiments use
- * for the outer learning rate ("a warm-up period ... followed by cosine
- * annealing", Appendix B):
+ * for the outer learning rate (Appendix B):
  *   t <  warmup : base * (start_factor + (1 - start_factor) * t / warmup)
  *   t >= warmup : kind 0: base
  *                 kind 1: min + (base - min) * (1 + cos(pi * tau / (total - warmup))) / 2,

@@ -71,7 +71,7 @@ typedef struct {
     uint64_t  n_outer;       /* outer syncs performed                              */
     double   *pow1, *pow2;   /* [K] beta1^s_k, beta2^s_k (running products)        */
     uint8_t  *last_b;        /* [K] decisions of the latest step                   */
-    /* global-norm gradient clipping (Appendix B: "gradient clipping enabled") */
+    /* global-norm gradient clipping (Appendix B: the GPT-Neo runs clip their gradients) */
     double    max_grad_norm; /* threshold; 0 = no clipping                         */
     const double *forced_sumsq; /* NULL, or [K] sums of squares to use instead of
                                 computing them (sampled replays of a large run)   */
@@ -302,8 +302,8 @@ void FN(outer_sync)(FN(state) *st)
     st->n_outer += 1;
 }
 
-/* DDP warm-up step (Sec. 3.3 "we initialize training with a DDP warm-up phase";
- * Sec. 4.1: Local SGD, DiLoCo and PALSGD all use DDP during the initial steps).
+/* DDP warm-up step (Sec. 3.3: training begins with a DDP phase; Sec. 4.1: Local SGD,
+ * DiLoCo and PALSGD all use DDP during the initial steps).
  * Mini-batch SGD over K workers: the gradients are averaged,
  *     gbar = (g_0 + g_1 + ... + g_{K-1}) / K      (ascending k, one division),
  * and every worker applies the same InnerOPT step with the plain step size

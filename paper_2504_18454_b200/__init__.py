@@ -25,8 +25,6 @@ from .binding import (  # noqa: F401
     TUNE_INNER_GRID_CAP,
     TUNE_OUTER_GRID_CAP,
     TUNE_INNER_VARIANT,
-    TUNE_PIPE_STAGES,
-    TUNE_CHUNK_MAJOR,
     TUNE_OUTER_SUB_ELEMS,
     TUNE_DDP_SUB_ELEMS,
     TUNE_DDP_VARIANT,

@@ -12,8 +12,8 @@ INNER_ADAMW, INNER_SGDM = 0, 1
 PREC_FP32, PREC_BF16_MASTER = 0, 1
 OUTER_SGD, OUTER_ADAMW = 0, 1
 SCHED_WARMUP_CONSTANT, SCHED_WARMUP_COSINE = 0, 1
-TUNE_INNER_GRID_CAP, TUNE_OUTER_GRID_CAP, TUNE_INNER_VARIANT, TUNE_PIPE_STAGES = 0, 1, 2, 3
-TUNE_CHUNK_MAJOR, TUNE_OUTER_SUB_ELEMS, TUNE_DDP_SUB_ELEMS, TUNE_DDP_VARIANT = 4, 5, 6, 7
+TUNE_INNER_GRID_CAP, TUNE_OUTER_GRID_CAP, TUNE_INNER_VARIANT = 0, 1, 2
+TUNE_OUTER_SUB_ELEMS, TUNE_DDP_SUB_ELEMS, TUNE_DDP_VARIANT = 5, 6, 7
 TUNE_OUTER_VARIANT, TUNE_OUTER_DYNAMIC = 8, 9
 MAX_WORKERS = 64
 
@@ -82,6 +82,14 @@ def lib() -> C.CDLL:
     L.palsgd_set_counters.argtypes = [vp, C.c_uint64, u64p, C.c_uint64, vp]
     L.palsgd_get_launch_count.argtypes = [vp, u64p]
     L.palsgd_set_tuning.argtypes = [vp, C.c_int, C.c_int64]
+    L.palsgd_exchange_numel.argtypes = [vp, u64p]
+    L.palsgd_set_worker_offset.argtypes = [vp, C.c_uint32]
+    L.palsgd_outer_partial.argtypes = [vp, vp, vp]
+    L.palsgd_outer_finish.argtypes = [vp, vp, C.c_uint32, vp]
+    for name in ("palsgd_exchange_numel", "palsgd_set_worker_offset", "palsgd_outer_partial", "palsgd_outer_finish"):
+        getattr(L, name).restype = C.c_int
+    L.palsgd_get_layout.argtypes = [vp, u64p, u64p, C.POINTER(C.c_uint32)]
+    L.palsgd_get_layout.restype = C.c_int
     L.palsgd_decision.argtypes = [C.c_uint64, C.c_uint64, C.c_uint32, C.c_double]
     for name in ("palsgd_init", "palsgd_inner_step", "palsgd_pseudo_sync", "palsgd_outer_sync",
                  "palsgd_step", "palsgd_step_host", "palsgd_get_counters", "palsgd_set_counters",
@@ -268,6 +276,27 @@ class Palsgd:
         n = C.c_uint64(0)
         self._check(lib().palsgd_get_launch_count(self._ctx, C.byref(n)), "palsgd_get_launch_count")
         return n.value
+
+    def exchange_numel(self) -> int:
+        n = C.c_uint64(0)
+        self._check(lib().palsgd_exchange_numel(self._ctx, C.byref(n)), "palsgd_exchange_numel")
+        return n.value
+
+    def set_worker_offset(self, k0: int) -> None:
+        self._check(lib().palsgd_set_worker_offset(self._ctx, int(k0)), "palsgd_set_worker_offset")
+
+    def outer_partial(self, exchange_ptr: int, stream: int = 0) -> None:
+        self._check(lib().palsgd_outer_partial(self._ctx, C.c_void_p(exchange_ptr), C.c_void_p(stream)),
+                    "palsgd_outer_partial")
+
+    def outer_finish(self, exchange_ptr: int, K_total: int, stream: int = 0) -> None:
+        self._check(lib().palsgd_outer_finish(self._ctx, C.c_void_p(exchange_ptr), int(K_total), C.c_void_p(stream)),
+                    "palsgd_outer_finish")
+
+    def get_layout(self):
+        ns, nc, ce = C.c_uint64(0), C.c_uint64(0), C.c_uint32(0)
+        self._check(lib().palsgd_get_layout(self._ctx, C.byref(ns), C.byref(nc), C.byref(ce)), "palsgd_get_layout")
+        return {"n_segments": ns.value, "n_chunks": nc.value, "chunk_elems": ce.value}
 
     def set_tuning(self, knob: int, value: int) -> None:
         self._check(lib().palsgd_set_tuning(self._ctx, knob, value), "palsgd_set_tuning")

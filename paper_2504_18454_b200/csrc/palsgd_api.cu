@@ -18,14 +18,23 @@
 
 #include "palsgd_kernels.cuh"
 #include "palsgd_norm.cuh"
-#include "palsgd_pipe.cuh"
 
 using namespace palsgd;
+
+// Default launch shapes of the outer-sync and DDP kernels (CTAs per SM of a persistent grid that draws
+// its items from a queue; 0 = one CTA per item), measured on B200.
+// A CTA that handles several items alternates between two stage buffers when both fit in this many bytes
+// (beyond it the second buffer would cost resident CTAs, which measured far worse than a drained stage).
+constexpr size_t kTwoStageLimit = 32 * 1024;
+constexpr int kOuterCtasPerSm = 0;
+constexpr int kDdpCtasPerSm = 4;
 
 struct Segment {
     size_t   first_tensor;
     size_t   n_tensors;
     uint64_t numel;
+    int      head;     // elements to peel off the front so that what follows is 16-byte aligned in every
+                       // buffer (0..7); -1 = no such count exists: the whole segment takes the scalar path
 };
 
 struct palsgd_ctx {
@@ -39,21 +48,24 @@ struct palsgd_ctx {
     // device tables
     void* d_blob = nullptr;                  // one allocation holding everything below
     Tables tb{};
+    // item tables of the outer-sync and DDP kernels (their own allocations: a tuning knob may rebuild them)
+    Chunk* d_oitems = nullptr;  uint32_t n_oitems = 0;
+    Chunk* d_ditems = nullptr;  uint32_t n_ditems = 0;
     uint64_t P = 0;
+    uint64_t exch_numel = 0;                 // floats in the exchange buffer of the multi-GPU outer sync
+    uint32_t k0 = 0;                         // the decision stream's index of local worker 0
     // host mirrors
     uint64_t t = 0, n_outer = 0, launches = 0;
     uint64_t thr = 0;
     int grid_cap_inner = 0, grid_cap_outer = 0;   // 0 = one CTA per work item
-    int inner_variant = 0;                        // launch shape of the inner kernel, 0 = default
-    int pipe_stages = 0;                          // ring depth of the pipelined kernel, 0 = as many as fit
-    int chunk_major = 0;                          // work-item order of the register-path inner kernel
+    int inner_variant = 0;                        // 0 = persistent grid + work queue (default), 18 = one CTA per item
     uint32_t chunk_elems = kChunkElems;           // elements per chunk-table entry (fixed at init)
     uint32_t outer_sub_elems = kOuterSubElems;    // elements per work item of the outer kernel
     uint32_t ddp_sub_elems = kDdpSubElems;        // elements per work item of the DDP warm-up kernel
     int ddp_variant = 0;                          // 0 = default, 1 = per-thread stores, 2 = staged bulk stores
     int outer_variant = 0;                        // the same for the outer kernel
     int outer_dynamic = -1;                       // outer / DDP kernels: CTAs per SM of a persistent grid, 0 = one CTA
-                                                  // per item, -1 = default (outer: 0, DDP: 4; measured)
+                                                  // per item, -1 = default (kOuterCtasPerSm / kDdpCtasPerSm)
     double max_grad_norm = 0.0;                   // global-norm clip threshold, 0 = off
     double outer_lr = 0.0;                        // OuterOPT learning rate of the next sync
     double opow1 = 1.0, opow2 = 1.0;              // outer_beta^n_outer (AdamW as OuterOPT), running products
@@ -63,6 +75,11 @@ struct palsgd_ctx {
     cudaGraphExec_t cycle_exec = nullptr;         // captured H-step cycle (palsgd_cycle_capture) or nullptr
     uint64_t cycle_launches = 0;                  // kernels inside one captured cycle
     int sm_count = 0, smem_optin = 0;             // device attributes read at init
+    // kernels whose dynamic-shared-memory limit has been raised on this context's device, with the limit set
+    std::vector<std::pair<const void*, int>> smem_attr;
+    bool failed = false;                          // a CUDA call failed midway through an earlier entry point:
+                                                  // device state and host mirrors may disagree, so every later
+                                                  // call that would touch them returns PALSGD_ESTATE
     std::string cuda_err;
 };
 
@@ -73,12 +90,16 @@ thread_local std::string g_noctx_err;
 int cuda_fail(palsgd_ctx* ctx, cudaError_t e, const char* what)
 {
     std::string msg = std::string(what) + ": " + cudaGetErrorString(e);
-    if (ctx) ctx->cuda_err = msg; else g_noctx_err = msg;
+    if (ctx) { ctx->cuda_err = msg; ctx->failed = true; } else g_noctx_err = msg;
     return PALSGD_ECUDA;
 }
 
 #define PALSGD_CUDA(ctx, call)                                            \
     do { cudaError_t e_ = (call); if (e_ != cudaSuccess) return cuda_fail((ctx), e_, #call); } while (0)
+
+// Entry points that read or advance the state refuse a context that an earlier CUDA failure left half-advanced.
+#define PALSGD_USABLE(ctx)                                                \
+    do { if (!(ctx)) return PALSGD_EINVAL; if ((ctx)->failed) return PALSGD_ESTATE; } while (0)
 
 inline bool finite_nonneg(double v) { return std::isfinite(v) && v >= 0.0; }
 inline size_t elem_size_param(int prec) { return prec == PALSGD_PREC_BF16_MASTER ? 2 : 4; }
@@ -143,6 +164,42 @@ unsigned grid_for(uint64_t n_items, int cap)
     return (unsigned)(g == 0 ? 1 : g);
 }
 
+// Cut every segment into pieces of at most `piece` elements (a multiple of 1024).  A segment whose
+// buffers all become 16-byte aligned after `head` elements gets those elements as one scalar piece
+// and vector pieces behind it; full vector pieces are listed first (the small ones fill the tail of
+// a launch instead of sitting between large ones).
+std::vector<Chunk> cut_segments(const std::vector<Segment>& segs, uint32_t piece)
+{
+    std::vector<Chunk> out;
+    for (size_t s = 0; s < segs.size(); ++s) {
+        const Segment& sg = segs[s];
+        uint64_t off = 0;
+        const bool vec = sg.head >= 0;
+        if (sg.head > 0) {
+            off = std::min<uint64_t>((uint64_t)sg.head, sg.numel);
+            out.push_back(Chunk{0, (uint32_t)off, (uint32_t)s});
+        }
+        for (; off < sg.numel; off += piece) {
+            const uint64_t len = std::min<uint64_t>(sg.numel - off, piece);
+            out.push_back(Chunk{off, (uint32_t)len, (uint32_t)s | (vec ? kSegVecFlag : 0u)});
+        }
+    }
+    auto is_full = [piece](const Chunk& c) { return (c.seg & kSegVecFlag) && c.len == piece; };
+    std::stable_partition(out.begin(), out.end(), is_full);
+    return out;
+}
+
+// (Re)build one of the item tables on the device.  Synchronous; frees the previous table.
+int upload_items(palsgd_ctx* ctx, const std::vector<Chunk>& items, Chunk** d_items, uint32_t* n_items)
+{
+    if (*d_items) { PALSGD_CUDA(ctx, cudaDeviceSynchronize()); cudaFree(*d_items); *d_items = nullptr; }
+    *n_items = (uint32_t)items.size();
+    if (items.empty()) return PALSGD_OK;
+    PALSGD_CUDA(ctx, cudaMalloc(reinterpret_cast<void**>(d_items), items.size() * sizeof(Chunk)));
+    PALSGD_CUDA(ctx, cudaMemcpy(*d_items, items.data(), items.size() * sizeof(Chunk), cudaMemcpyHostToDevice));
+    return PALSGD_OK;
+}
+
 OuterArgs outer_args(const palsgd_ctx* ctx)
 {
     OuterArgs a{};
@@ -162,76 +219,28 @@ OuterArgs outer_args(const palsgd_ctx* ctx)
         a.odecay = (float)(1.0 - ctx->outer_lr * c.outer_weight_decay);
         a.oeps = (float)c.outer_eps;
     }
+    a.items = ctx->d_oitems;
+    a.n_items = ctx->n_oitems;
     a.sub_elems = ctx->outer_sub_elems;
-    a.parts = (ctx->chunk_elems + a.sub_elems - 1) / a.sub_elems;
+    a.n_stage = 1;
     return a;
 }
 
-// Launch shapes of the fused inner kernel: U = 128-bit loads in flight per
-// stream and thread, MINB = CTAs per SM the register budget is held to.
-template <int INNER, int PREC>
-void launch_inner_variant(int variant, unsigned grid, cudaStream_t s, const InnerArgs& a)
+// Raise a kernel's dynamic-shared-memory limit once per context (the attribute belongs to the
+// function on the context's device; setting it again on every launch costs a few microseconds).
+int ensure_dyn_smem(palsgd_ctx* ctx, const void* kernel, size_t bytes)
 {
-    switch (variant) {
-        case 1:  palsgd_inner_kernel<INNER, PREC, 1, 4><<<grid, kThreads, 0, s>>>(a); break;
-        case 2:  palsgd_inner_kernel<INNER, PREC, 1, 3><<<grid, kThreads, 0, s>>>(a); break;
-        case 3:  palsgd_inner_kernel<INNER, PREC, 2, 2><<<grid, kThreads, 0, s>>>(a); break;
-        case 4:  palsgd_inner_kernel<INNER, PREC, 2, 3><<<grid, kThreads, 0, s>>>(a); break;
-        case 5:  palsgd_inner_kernel<INNER, PREC, 4, 1><<<grid, kThreads, 0, s>>>(a); break;
-        case 6:  palsgd_inner_kernel<INNER, PREC, 1, 6><<<grid, kThreads, 0, s>>>(a); break;
-        case 7:  palsgd_inner_kernel<INNER, PREC, 0, 6><<<grid, kThreads, 0, s>>>(a); break;
-        case 8:  palsgd_inner_kernel<INNER, PREC, 0, 5><<<grid, kThreads, 0, s>>>(a); break;
-        case 9:  palsgd_inner_kernel<INNER, PREC, 0, 8><<<grid, kThreads, 0, s>>>(a); break;
-        case 13: palsgd_inner_kernel<INNER, PREC, -1, 4><<<grid, kThreads, 0, s>>>(a); break;
-        case 14: palsgd_inner_kernel<INNER, PREC, -1, 3><<<grid, kThreads, 0, s>>>(a); break;
-        case 15: palsgd_inner_kernel<INNER, PREC, -1, 5><<<grid, kThreads, 0, s>>>(a); break;
-        default:      // measured best on B200: one 128-bit load per stream and thread, many CTAs per SM
-            if (PREC) palsgd_inner_kernel<INNER, PREC, 1, 4><<<grid, kThreads, 0, s>>>(a);
-            else      palsgd_inner_kernel<INNER, PREC, 1, 6><<<grid, kThreads, 0, s>>>(a);
-            break;
-    }
-}
-
-using PipeKernel = void (*)(const InnerArgs, uint32_t, uint32_t);
-template <int INNER, int PREC, int NC>
-PipeKernel pipe_kernel_ptr()
-{
-    if constexpr (NC == 0) return palsgd_inner_pipe_all_kernel<INNER, PREC>;
-    else return palsgd_inner_pipe_kernel<INNER, PREC, NC>;
-}
-
-// Persistent TMA-ring kernel: one CTA per SM, as many stages as shared memory holds.
-template <int INNER, int PREC, int NC>
-int launch_inner_pipe(palsgd_ctx* ctx, const InnerArgs& a, cudaStream_t s)
-{
-    constexpr uint32_t stage_bytes = ((INNER == 0 ? 12u : 8u) + (PREC ? 2u : 4u)) * kStageElems;
-    const int budget = ctx->smem_optin - 4096;              // static shared memory and the system's share
-    int stages = std::min<int>(kPipeMaxStages, budget / (int)stage_bytes);
-    if (ctx->pipe_stages > 0) stages = std::min(stages, ctx->pipe_stages);
-    if (stages < 2) return PALSGD_EUNSUPPORTED;
-    const size_t dyn = (size_t)stages * stage_bytes;
-    auto kernel = pipe_kernel_ptr<INNER, PREC, NC>();
-    constexpr unsigned threads = NC == 0 ? 1024u : (unsigned)NC + 32u;
-    static int attr_for_device = -1;                         // opt in to large dynamic shared memory once
-    int dev = 0;
-    PALSGD_CUDA(ctx, cudaGetDevice(&dev));
-    if (attr_for_device != dev) {
-        PALSGD_CUDA(ctx, cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, budget));
-        attr_for_device = dev;
-    }
-    const uint64_t n_items = (uint64_t)ctx->tb.n_full * ctx->cfg.K * (ctx->chunk_elems / kStageElems);
-    const int cap = ctx->grid_cap_inner > 0 ? ctx->grid_cap_inner : ctx->sm_count;
-    const unsigned grid = grid_for(n_items, cap);
-    return launch_checked(ctx, [&] { kernel<<<grid, threads, dyn, s>>>(a, (uint32_t)stages, stage_bytes); });
-}
-
-// NC = 0 selects the form in which all 1024 threads consume and thread 0 also produces.
-template <int INNER, int PREC>
-int launch_inner_pipe_nc(palsgd_ctx* ctx, int variant, const InnerArgs& a, cudaStream_t s)
-{
-    if (variant == 11) return launch_inner_pipe<INNER, PREC, 256>(ctx, a, s);
-    if (variant == 10) return launch_inner_pipe<INNER, PREC, 512>(ctx, a, s);
-    return launch_inner_pipe<INNER, PREC, 0>(ctx, a, s);
+    if (bytes + 4096 <= 48 * 1024) return PALSGD_OK;         // static + dynamic within the default limit
+    for (auto& kv : ctx->smem_attr)
+        if (kv.first == kernel) {
+            if (kv.second >= (int)bytes) return PALSGD_OK;
+            PALSGD_CUDA(ctx, cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes));
+            kv.second = (int)bytes;
+            return PALSGD_OK;
+        }
+    PALSGD_CUDA(ctx, cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes));
+    ctx->smem_attr.emplace_back(kernel, (int)bytes);
+    return PALSGD_OK;
 }
 
 // Norm pass of the gradient clip: per-worker norms (ddp = false) or the norm of the averaged gradient.
@@ -243,6 +252,7 @@ int launch_gradnorm(palsgd_ctx* ctx, bool ddp, cudaStream_t s)
     a.thr = ctx->thr;
     a.max_norm = ctx->max_grad_norm;
     a.Kf = (float)ctx->cfg.K;
+    a.k0 = ctx->k0;
     a.ddp = ddp ? 1u : 0u;
     // chunks per work item: up to 8 (4 for the K-stream averaged form), fewer while that would leave
     // under ~2048 items; fixed by the problem, so results never depend on the device or on tuning knobs
@@ -258,40 +268,29 @@ int launch_gradnorm(palsgd_ctx* ctx, bool ddp, cudaStream_t s)
     });
 }
 
+// Launch shape of the fused inner kernel, measured on B200: one 128-bit load per stream and thread,
+// registers held to 4 (mixed precision) or 6 (fp32) CTAs per SM.
 int launch_inner(palsgd_ctx* ctx, const InnerArgs& a, cudaStream_t s)
 {
-    // the shared-memory-ring forms do not carry the clip coefficient: clipped steps take the register path
     const bool whole_step = a.k_begin == 0 && a.k_count == ctx->cfg.K && a.tick;
-    if (whole_step && !a.clip_on && ctx->inner_variant >= 10 && ctx->inner_variant <= 12 && ctx->tb.n_full > 0 &&
-        ctx->chunk_elems % kStageElems == 0) {
-        const bool adam_ = ctx->cfg.inner == PALSGD_INNER_ADAMW;
-        const bool bf_ = ctx->cfg.precision == PALSGD_PREC_BF16_MASTER;
-        const int v_ = ctx->inner_variant;
-        if (adam_ && !bf_)  return launch_inner_pipe_nc<0, 0>(ctx, v_, a, s);
-        if (!adam_ && !bf_) return launch_inner_pipe_nc<1, 0>(ctx, v_, a, s);
-        if (adam_ && bf_)   return launch_inner_pipe_nc<0, 1>(ctx, v_, a, s);
-        return launch_inner_pipe_nc<1, 1>(ctx, v_, a, s);
-    }
     const uint64_t n_items = (uint64_t)ctx->tb.n_chunks * a.k_count;
     const bool adam = ctx->cfg.inner == PALSGD_INNER_ADAMW;
     const bool bf = ctx->cfg.precision == PALSGD_PREC_BF16_MASTER;
-    int v = ctx->inner_variant;
     InnerArgs b = a;
     // with nothing to stream a one-CTA launch still advances the counters
     unsigned grid = grid_for(n_items, ctx->grid_cap_inner);
     // Default: a persistent grid (as many CTAs as are resident at once) that draws its work items from a queue
     // in device memory -- no tail of idle SMs, one prologue per CTA (measured +0.5 .. +6 % over one CTA per
-    // item, most on small models).  Variant 18 = the default shape with one CTA per item.
-    if (v == 0 && whole_step && ctx->sm_count > 0 && ctx->grid_cap_inner == 0) {
+    // item, most on small models).  Variant 18 = the same shape with one CTA per item.
+    if (ctx->inner_variant != 18 && whole_step && ctx->sm_count > 0 && ctx->grid_cap_inner == 0) {
         b.dynamic = 1;
         grid = grid_for(n_items, ctx->sm_count * (bf ? 4 : 6));
     }
-    if (v == 18) v = 0;
     return launch_checked(ctx, [&] {
-        if (adam && !bf)       launch_inner_variant<0, 0>(v, grid, s, b);
-        else if (!adam && !bf) launch_inner_variant<1, 0>(v, grid, s, b);
-        else if (adam && bf)   launch_inner_variant<0, 1>(v, grid, s, b);
-        else                   launch_inner_variant<1, 1>(v, grid, s, b);
+        if (adam && !bf)       palsgd_inner_kernel<0, 0, 1, 6><<<grid, kThreads, 0, s>>>(b);
+        else if (!adam && !bf) palsgd_inner_kernel<1, 0, 1, 6><<<grid, kThreads, 0, s>>>(b);
+        else if (adam && bf)   palsgd_inner_kernel<0, 1, 1, 4><<<grid, kThreads, 0, s>>>(b);
+        else                   palsgd_inner_kernel<1, 1, 1, 4><<<grid, kThreads, 0, s>>>(b);
     });
 }
 
@@ -375,44 +374,47 @@ extern "C" int palsgd_init(palsgd_ctx** out, const palsgd_config* cfg, size_t n_
         return ga + numel[j] * 4 == reinterpret_cast<const char*>(bufs->global[j + 1]) &&
                ua + numel[j] * 4 == reinterpret_cast<const char*>(bufs->outer_mom[j + 1]);
     };
+    // Elements to peel off a segment's front so that the rest is 16-byte aligned in every buffer: h with
+    // (address + h * element size) % 16 == 0 for all of them (0 for buffers that are aligned already,
+    // 7 for a packed list shifted by one element: fp32 at +4 bytes, bf16 at +2).  -1 if there is none.
+    auto head_of = [&](size_t first) {
+        for (int h = 0; h < 8; ++h) {
+            bool ok = aligned(reinterpret_cast<const char*>(bufs->global[first]) + 4 * h, 16) &&
+                      aligned(reinterpret_cast<const char*>(bufs->outer_mom[first]) + 4 * h, 16) &&
+                      (!oadam || aligned(reinterpret_cast<const char*>(bufs->outer_v[first]) + 4 * h, 16));
+            for (uint32_t k = 0; k < K && ok; ++k)
+                for (const Kind& kd : kinds)
+                    if (kd.present && !aligned(static_cast<const char*>(buf_ptr(bufs, kd.id, (size_t)k * n_tensors + first)) +
+                                                   kd.esize * h, 16))
+                        ok = false;
+            if (ok) return h;
+        }
+        return -1;
+    };
     for (size_t j = 0; j < n_tensors;) {
-        Segment sg{j, 1, numel[j]};
+        Segment sg{j, 1, numel[j], 0};
         while (sg.first_tensor + sg.n_tensors < n_tensors &&
                adjacent(sg.first_tensor + sg.n_tensors - 1)) {
             sg.numel += numel[sg.first_tensor + sg.n_tensors];
             sg.n_tensors += 1;
         }
         j += sg.n_tensors;
-        if (sg.numel > 0) ctx->segs.push_back(sg);
+        // (an empty tensor between two adjacent ones is skipped over by the fusion above; the first
+        //  tensor of a non-empty segment may itself be empty, its pointer still marks the start)
+        if (sg.numel > 0) { sg.head = head_of(sg.first_tensor); ctx->segs.push_back(sg); }
     }
     const size_t n_seg = ctx->segs.size();
 
-    // ---- chunk table and per-segment vector-path flag
+    // ---- chunk table of the inner kernel; item tables of the outer-sync and DDP kernels
     // Elements per inner work item, measured best on B200: 4096 for fp32 AdamW, 8192 otherwise.
     ctx->chunk_elems = (!bf && adam) ? 4096u : kChunkElems;
-    if (const char* e = std::getenv("PALSGD_CHUNK_ELEMS")) {      // tuning aid: a multiple of 1024
-        const long v = std::atol(e);
-        if (v >= 1024 && v <= (1 << 20) && v % 1024 == 0) ctx->chunk_elems = (uint32_t)v;
+    const std::vector<Chunk> chunks = cut_segments(ctx->segs, ctx->chunk_elems);
+    const std::vector<Chunk> oitems = cut_segments(ctx->segs, ctx->outer_sub_elems);
+    const std::vector<Chunk> ditems = cut_segments(ctx->segs, ctx->ddp_sub_elems);
+    if (chunks.size() > 0x7FFFFFFFull / K || oitems.size() > 0x7FFFFFFFull || ditems.size() > 0x7FFFFFFFull) {
+        delete ctx;
+        return PALSGD_EUNSUPPORTED;
     }
-    std::vector<Chunk> chunks;
-    for (size_t s = 0; s < n_seg; ++s) {
-        const Segment& sg = ctx->segs[s];
-        bool vec = aligned(bufs->global[sg.first_tensor], 16) && aligned(bufs->outer_mom[sg.first_tensor], 16) &&
-                   (!oadam || aligned(bufs->outer_v[sg.first_tensor], 16));
-        for (uint32_t k = 0; k < K && vec; ++k)
-            for (const Kind& kd : kinds)
-                if (kd.present && !aligned(buf_ptr(bufs, kd.id, (size_t)k * n_tensors + sg.first_tensor), 16))
-                    vec = false;
-        for (uint64_t off = 0; off < sg.numel; off += ctx->chunk_elems) {
-            const uint64_t len = sg.numel - off < ctx->chunk_elems ? sg.numel - off : ctx->chunk_elems;
-            chunks.push_back(Chunk{off, (uint32_t)len, (uint32_t)s | (vec ? kSegVecFlag : 0u)});
-        }
-    }
-    if (chunks.size() > 0x7FFFFFFFull / K) { delete ctx; return PALSGD_EUNSUPPORTED; }
-    // full, aligned chunks first: the pipelined kernel streams exactly those through shared memory
-    const uint32_t full_len = ctx->chunk_elems;
-    auto is_full = [full_len](const Chunk& c) { return (c.seg & kSegVecFlag) && c.len == full_len; };
-    const size_t n_full = std::stable_partition(chunks.begin(), chunks.end(), is_full) - chunks.begin();
 
     // ---- one device blob: [DevState][chunks][7 pointer tables]
     const size_t per_slot = (size_t)K * n_seg * sizeof(void*);
@@ -420,7 +422,7 @@ extern "C" int palsgd_init(palsgd_ctx** out, const palsgd_config* cfg, size_t n_
     size_t off_state = 0;
     size_t off_chunks = round_up(sizeof(DevState), 256);
     size_t off_tabs = round_up(off_chunks + chunks.size() * sizeof(Chunk), 256);
-    const size_t off_norm = off_tabs + 5 * round_up(per_slot, 256) + 3 * round_up(per_seg, 256) + 256;
+    const size_t off_norm = off_tabs + 5 * round_up(per_slot, 256) + 4 * round_up(per_seg, 256) + 256;
     const size_t total = off_norm + round_up(chunks.size() * K * sizeof(double2), 256) + 256;
     std::vector<char> host(total, 0);
     DevState hs{};
@@ -468,7 +470,6 @@ extern "C" int palsgd_init(palsgd_ctx** out, const palsgd_config* cfg, size_t n_
     tb.n_chunks = (uint32_t)chunks.size();
     tb.n_seg = (uint32_t)n_seg;
     tb.K = K;
-    tb.n_full = (uint32_t)n_full;
     tb.chunk_elems = ctx->chunk_elems;
     void* t_param = fill_slot_table(0);
     tb.grad = static_cast<const void* const*>(fill_slot_table(1));
@@ -480,11 +481,24 @@ extern "C" int palsgd_init(palsgd_ctx** out, const palsgd_config* cfg, size_t n_
     tb.outer_v = oadam ? static_cast<float* const*>(fill_seg_table(bufs->outer_v)) : nullptr;
     tb.xf = static_cast<float* const*>(bf ? t_master : t_param);
     tb.xw = bf ? static_cast<__nv_bfloat16* const*>(t_param) : nullptr;
+    {   // exchange-buffer offsets: the buffer is the tensor list packed back to back (a function of the
+        // element counts alone, so that every GPU of a job lays it out alike whatever its memory layout)
+        uint64_t* h = reinterpret_cast<uint64_t*>(host.data() + cur);
+        std::vector<uint64_t> prefix(n_tensors + 1, 0);
+        for (size_t j = 0; j < n_tensors; ++j) prefix[j + 1] = prefix[j] + numel[j];
+        for (size_t sgi = 0; sgi < n_seg; ++sgi) h[sgi] = prefix[ctx->segs[sgi].first_tensor];
+        ctx->exch_numel = P;
+        tb.exch_off = reinterpret_cast<const uint64_t*>(d + cur);
+        cur += round_up(per_seg, 256);
+    }
     tb.norm_part = reinterpret_cast<double2*>(d + off_norm);
 
     cudaError_t e = cudaMemcpyAsync(ctx->d_blob, host.data(), total, cudaMemcpyHostToDevice, s);
     if (e == cudaSuccess) e = cudaStreamSynchronize(s);      // `host` is pageable and dies with this scope
     if (e != cudaSuccess) { rc = cuda_fail(nullptr, e, "table upload"); cudaFree(ctx->d_blob); delete ctx; return rc; }
+    rc = upload_items(ctx, oitems, &ctx->d_oitems, &ctx->n_oitems);
+    if (rc == PALSGD_OK) rc = upload_items(ctx, ditems, &ctx->d_ditems, &ctx->n_ditems);
+    if (rc) { g_noctx_err = ctx->cuda_err; palsgd_destroy(ctx); return rc == PALSGD_ECUDA ? rc : PALSGD_ENOMEM; }
 
     if (tb.n_chunks > 0) {
         const OuterArgs oa = outer_args(ctx);
@@ -493,7 +507,7 @@ extern "C" int palsgd_init(palsgd_ctx** out, const palsgd_config* cfg, size_t n_
             if (bf) palsgd_init_kernel<1><<<grid, kThreads, 0, s>>>(oa, adam ? 1 : 0);
             else    palsgd_init_kernel<0><<<grid, kThreads, 0, s>>>(oa, adam ? 1 : 0);
         });
-        if (rc) { g_noctx_err = ctx->cuda_err; cudaFree(ctx->d_blob); delete ctx; return rc; }
+        if (rc) { g_noctx_err = ctx->cuda_err; palsgd_destroy(ctx); return rc; }
     }
     *out = ctx;
     return PALSGD_OK;
@@ -523,18 +537,18 @@ static InnerArgs inner_args(const palsgd_ctx* ctx, double lr_t, double eta_t)
     a.decay = (float)(1.0 - lr_d * c.weight_decay);
     a.mu = (float)c.momentum;
     a.wd = (float)c.weight_decay;
-    a.chunk_major = (uint32_t)ctx->chunk_major;
     // clipped gradients: one norm pass first (not needed when every worker pulls)
     a.clip_on = (ctx->max_grad_norm > 0.0 && c.p < 1.0) ? 1u : 0u;
     a.k_begin = 0;
     a.k_count = c.K;
+    a.k0 = ctx->k0;
     a.tick = 1;
     return a;
 }
 
 extern "C" int palsgd_inner_step(palsgd_ctx* ctx, double lr_t, double eta_t, void* stream)
 {
-    if (!ctx) return PALSGD_EINVAL;
+    PALSGD_USABLE(ctx);
     if (!finite_nonneg(lr_t) || !finite_nonneg(eta_t)) return PALSGD_EINVAL;
     const InnerArgs a = inner_args(ctx, lr_t, eta_t);
     int rc = PALSGD_OK;
@@ -547,7 +561,7 @@ extern "C" int palsgd_inner_step(palsgd_ctx* ctx, double lr_t, double eta_t, voi
 
 extern "C" int palsgd_ddp_step(palsgd_ctx* ctx, double lr_t, void* stream)
 {
-    if (!ctx) return PALSGD_EINVAL;
+    PALSGD_USABLE(ctx);
     if (!finite_nonneg(lr_t)) return PALSGD_EINVAL;
     const palsgd_config& c = ctx->cfg;
     DdpArgs a{};
@@ -564,18 +578,27 @@ extern "C" int palsgd_ddp_step(palsgd_ctx* ctx, double lr_t, void* stream)
     a.mu = (float)c.momentum;
     a.wd = (float)c.weight_decay;
     a.Kf = (float)c.K;
+    a.items = ctx->d_ditems;
+    a.n_items = ctx->n_ditems;
     a.sub_elems = ctx->ddp_sub_elems;
-    a.parts = (ctx->chunk_elems + a.sub_elems - 1) / a.sub_elems;
-    // with nothing to stream a one-CTA launch still advances the counters
-    const unsigned grid = grid_for((uint64_t)ctx->tb.n_chunks * a.parts, ctx->grid_cap_outer);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const bool adam = c.inner == PALSGD_INNER_ADAMW;
     const bool bf = c.precision == PALSGD_PREC_BF16_MASTER;
     a.clip_on = ctx->max_grad_norm > 0.0 ? 1u : 0u;
     int rc = PALSGD_OK;
     if (a.clip_on) { rc = launch_gradnorm(ctx, true, s); if (rc) return rc; }
-    // staged form: new state in shared memory, fanned out to the K slots by bulk asynchronous stores
-    const size_t stage_bytes = (size_t)a.sub_elems * ((adam ? 12u : 8u) + (bf ? 2u : 0u));
+    // with nothing to stream a one-CTA launch still advances the counters
+    unsigned grid = grid_for(a.n_items, ctx->grid_cap_outer);
+    const int dyn = ctx->outer_dynamic < 0 ? kDdpCtasPerSm : ctx->outer_dynamic;
+    if (dyn && ctx->grid_cap_outer == 0 && ctx->sm_count > 0) {                      // persistent grid + work queue
+        a.dynamic = 1;
+        grid = grid_for(a.n_items, ctx->sm_count * dyn);
+    }
+    // staged form: new state in shared memory, fanned out to the K slots by bulk asynchronous stores; a CTA
+    // that handles several items alternates between two stage buffers
+    const size_t one_stage = (size_t)a.sub_elems * ((adam ? 12u : 8u) + (bf ? 2u : 0u));
+    a.n_stage = (grid < a.n_items && 2 * one_stage <= kTwoStageLimit) ? 2u : 1u;
+    const size_t stage_bytes = one_stage * a.n_stage;
     const bool bcast = ctx->ddp_variant != 1 && (int)stage_bytes <= ctx->smem_optin - 4096;   // measured best
     using DdpKernel = void (*)(const DdpArgs);
     DdpKernel kernel;
@@ -583,15 +606,8 @@ extern "C" int palsgd_ddp_step(palsgd_ctx* ctx, double lr_t, void* stream)
                              : (bf ? palsgd_ddp_kernel<1, 1, 1> : palsgd_ddp_kernel<1, 0, 1>);
     else       kernel = adam ? (bf ? palsgd_ddp_kernel<0, 1, 0> : palsgd_ddp_kernel<0, 0, 0>)
                              : (bf ? palsgd_ddp_kernel<1, 1, 0> : palsgd_ddp_kernel<1, 0, 0>);
-    if (bcast && stage_bytes + 4096 > 48 * 1024)   // static + dynamic above the default limit: opt in (idempotent)
-        PALSGD_CUDA(ctx, cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)stage_bytes));
-    unsigned g = grid;
-    const int dyn = ctx->outer_dynamic < 0 ? 4 : ctx->outer_dynamic;
-    if (dyn && ctx->grid_cap_outer == 0 && ctx->sm_count > 0) {                      // persistent grid + work queue
-        a.dynamic = 1;
-        g = grid_for((uint64_t)ctx->tb.n_chunks * a.parts, ctx->sm_count * dyn);
-    }
-    rc = launch_checked(ctx, [&] { kernel<<<g, kThreads, bcast ? stage_bytes : 0, s>>>(a); });
+    if (bcast) { rc = ensure_dyn_smem(ctx, reinterpret_cast<const void*>(kernel), stage_bytes); if (rc) return rc; }
+    rc = launch_checked(ctx, [&] { kernel<<<grid, kThreads, bcast ? stage_bytes : 0, s>>>(a); });
     if (rc) return rc;
     ctx->t += 1;
     return PALSGD_OK;
@@ -599,7 +615,8 @@ extern "C" int palsgd_ddp_step(palsgd_ctx* ctx, double lr_t, void* stream)
 
 extern "C" int palsgd_pseudo_sync(palsgd_ctx* ctx, uint64_t worker_mask, double beta, void* stream)
 {
-    if (!ctx || !std::isfinite(beta)) return PALSGD_EINVAL;
+    PALSGD_USABLE(ctx);
+    if (!std::isfinite(beta)) return PALSGD_EINVAL;
     const uint32_t K = ctx->cfg.K;
     if (K < 64 && (worker_mask >> K) != 0) return PALSGD_EINVAL;
     if (worker_mask == 0 || ctx->tb.n_chunks == 0) return PALSGD_OK;
@@ -618,15 +635,23 @@ extern "C" int palsgd_pseudo_sync(palsgd_ctx* ctx, uint64_t worker_mask, double 
 
 extern "C" int palsgd_outer_sync(palsgd_ctx* ctx, void* stream)
 {
-    if (!ctx) return PALSGD_EINVAL;
-    if (ctx->tb.n_chunks > 0) {
-        const OuterArgs a = outer_args(ctx);
-        const unsigned grid = grid_for((uint64_t)ctx->tb.n_chunks * a.parts, ctx->grid_cap_outer);
+    PALSGD_USABLE(ctx);
+    if (ctx->n_oitems > 0) {
+        OuterArgs a = outer_args(ctx);
         cudaStream_t s = static_cast<cudaStream_t>(stream);
         const bool bf = ctx->cfg.precision == PALSGD_PREC_BF16_MASTER;
         const bool oadam = ctx->cfg.outer_opt == PALSGD_OUTER_ADAMW;
-        // staged form: new x_g (and u, bf16 copy) in shared memory, K slots written by bulk asynchronous stores
-        const size_t stage_bytes = (size_t)a.sub_elems * (8u + (oadam ? 4u : 0u) + (bf ? 2u : 0u));
+        unsigned grid = grid_for(a.n_items, ctx->grid_cap_outer);
+        const int dyn = ctx->outer_dynamic < 0 ? kOuterCtasPerSm : ctx->outer_dynamic;
+        if (dyn && ctx->grid_cap_outer == 0 && ctx->sm_count > 0) {                  // persistent grid + work queue
+            a.dynamic = 1;
+            grid = grid_for(a.n_items, ctx->sm_count * dyn);
+        }
+        // staged form: new x_g (and u, bf16 copy) in shared memory, K slots written by bulk asynchronous stores;
+        // a CTA that handles several items alternates between two stage buffers
+        const size_t one_stage = (size_t)a.sub_elems * (8u + (oadam ? 4u : 0u) + (bf ? 2u : 0u));
+        a.n_stage = (grid < a.n_items && 2 * one_stage <= kTwoStageLimit) ? 2u : 1u;
+        const size_t stage_bytes = one_stage * a.n_stage;
         const bool bcast = ctx->outer_variant != 1 && (int)stage_bytes <= ctx->smem_optin - 4096;   // measured best
         using OuterKernel = void (*)(const OuterArgs);
         OuterKernel kernel;
@@ -634,16 +659,72 @@ extern "C" int palsgd_outer_sync(palsgd_ctx* ctx, void* stream)
                                : (oadam ? palsgd_outer_kernel<0, 1, 1> : palsgd_outer_kernel<0, 0, 1>);
         else       kernel = bf ? (oadam ? palsgd_outer_kernel<1, 1, 0> : palsgd_outer_kernel<1, 0, 0>)
                                : (oadam ? palsgd_outer_kernel<0, 1, 0> : palsgd_outer_kernel<0, 0, 0>);
-        if (bcast && stage_bytes + 4096 > 48 * 1024)
-            PALSGD_CUDA(ctx, cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)stage_bytes));
-        OuterArgs b = a;
-        unsigned g = grid;
-        const int dyn = ctx->outer_dynamic < 0 ? 0 : ctx->outer_dynamic;
-        if (dyn && ctx->grid_cap_outer == 0 && ctx->sm_count > 0) {                  // persistent grid + work queue
-            b.dynamic = 1;
-            g = grid_for((uint64_t)ctx->tb.n_chunks * a.parts, ctx->sm_count * dyn);
-        }
-        int rc = launch_checked(ctx, [&] { kernel<<<g, kThreads, bcast ? stage_bytes : 0, s>>>(b); });
+        if (bcast) { const int rc = ensure_dyn_smem(ctx, reinterpret_cast<const void*>(kernel), stage_bytes); if (rc) return rc; }
+        int rc = launch_checked(ctx, [&] { kernel<<<grid, kThreads, bcast ? stage_bytes : 0, s>>>(a); });
+        if (rc) return rc;
+    }
+    if (ctx->cfg.outer_opt == PALSGD_OUTER_ADAMW) {
+        ctx->opow1 *= ctx->cfg.outer_beta1;
+        ctx->opow2 *= ctx->cfg.outer_beta2;
+    }
+    ctx->n_outer += 1;
+    return PALSGD_OK;
+}
+
+// ------------------------------------------------------------------------- outer sync over several GPUs
+
+extern "C" int palsgd_exchange_numel(palsgd_ctx* ctx, uint64_t* n_floats)
+{
+    if (!ctx || !n_floats) return PALSGD_EINVAL;
+    *n_floats = ctx->exch_numel;
+    return PALSGD_OK;
+}
+
+extern "C" int palsgd_set_worker_offset(palsgd_ctx* ctx, uint32_t k0)
+{
+    PALSGD_USABLE(ctx);
+    if ((uint64_t)k0 + ctx->cfg.K > 0xFFFFFFFFull) return PALSGD_EINVAL;
+    ctx->k0 = k0;
+    return PALSGD_OK;
+}
+
+extern "C" int palsgd_outer_partial(palsgd_ctx* ctx, float* exchange, void* stream)
+{
+    PALSGD_USABLE(ctx);
+    if (!exchange && ctx->exch_numel > 0) return PALSGD_EINVAL;
+    if (!aligned(exchange, 16)) return PALSGD_EALIGN;
+    if (ctx->n_oitems == 0) return PALSGD_OK;
+    OuterArgs a = outer_args(ctx);
+    a.sum_out = exchange;
+    const unsigned grid = grid_for(a.n_items, ctx->grid_cap_outer);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    return launch_checked(ctx, [&] { palsgd_outer_partial_kernel<8><<<grid, kThreads, 0, s>>>(a); });
+}
+
+extern "C" int palsgd_outer_finish(palsgd_ctx* ctx, const float* exchange, uint32_t K_total, void* stream)
+{
+    PALSGD_USABLE(ctx);
+    if (K_total < ctx->cfg.K) return PALSGD_EINVAL;
+    if (!exchange && ctx->exch_numel > 0) return PALSGD_EINVAL;
+    if (!aligned(exchange, 16)) return PALSGD_EALIGN;
+    if (ctx->n_oitems > 0) {
+        OuterArgs a = outer_args(ctx);
+        a.sum_in = exchange;
+        a.Kf = (float)K_total;
+        cudaStream_t s = static_cast<cudaStream_t>(stream);
+        const bool bf = ctx->cfg.precision == PALSGD_PREC_BF16_MASTER;
+        const bool oadam = ctx->cfg.outer_opt == PALSGD_OUTER_ADAMW;
+        const unsigned grid = grid_for(a.n_items, ctx->grid_cap_outer);
+        const size_t one_stage = (size_t)a.sub_elems * (8u + (oadam ? 4u : 0u) + (bf ? 2u : 0u));
+        a.n_stage = (grid < a.n_items && 2 * one_stage <= kTwoStageLimit) ? 2u : 1u;
+        const size_t stage_bytes = one_stage * a.n_stage;
+        if ((int)stage_bytes > ctx->smem_optin - 4096) return PALSGD_EUNSUPPORTED;   // an item size set far too large
+        using OuterKernel = void (*)(const OuterArgs);
+        OuterKernel kernel = bf ? (oadam ? palsgd_outer_kernel<1, 1, 1, 1> : palsgd_outer_kernel<1, 0, 1, 1>)
+                                : (oadam ? palsgd_outer_kernel<0, 1, 1, 1> : palsgd_outer_kernel<0, 0, 1, 1>);
+        int rc = ensure_dyn_smem(ctx, reinterpret_cast<const void*>(kernel), stage_bytes);
+        if (rc) return rc;
+        rc = launch_checked(ctx, [&] { kernel<<<grid, kThreads, stage_bytes, s>>>(a); });
         if (rc) return rc;
     }
     if (ctx->cfg.outer_opt == PALSGD_OUTER_ADAMW) {
@@ -666,7 +747,7 @@ extern "C" int palsgd_step(palsgd_ctx* ctx, double lr_t, double eta_t, void* str
 
 extern "C" int palsgd_cycle_capture(palsgd_ctx* ctx, double lr_t, double eta_t)
 {
-    if (!ctx) return PALSGD_EINVAL;
+    PALSGD_USABLE(ctx);
     if (!finite_nonneg(lr_t) || !finite_nonneg(eta_t)) return PALSGD_EINVAL;
     if (ctx->t % ctx->cfg.H != 0) return PALSGD_ESTATE;             // a cycle starts right after a sync
     if (ctx->cfg.outer_opt == PALSGD_OUTER_ADAMW) return PALSGD_EUNSUPPORTED;   // its scalars change every round
@@ -698,7 +779,7 @@ extern "C" int palsgd_cycle_capture(palsgd_ctx* ctx, double lr_t, double eta_t)
 
 extern "C" int palsgd_cycle_launch(palsgd_ctx* ctx, void* stream)
 {
-    if (!ctx) return PALSGD_EINVAL;
+    PALSGD_USABLE(ctx);
     if (!ctx->cycle_exec || ctx->t % ctx->cfg.H != 0) return PALSGD_ESTATE;
     PALSGD_CUDA(ctx, cudaGraphLaunch(ctx->cycle_exec, static_cast<cudaStream_t>(stream)));
     ctx->t += ctx->cfg.H;
@@ -710,22 +791,28 @@ extern "C" int palsgd_cycle_launch(palsgd_ctx* ctx, void* stream)
 extern "C" int palsgd_step_host(palsgd_ctx* ctx, const void* const* h_grad, double lr_t, double eta_t,
                                 float* const* h_global, uint8_t* h_decisions, int* synced, void* stream)
 {
-    if (!ctx || !h_grad) return PALSGD_EINVAL;
+    PALSGD_USABLE(ctx);
+    if (!h_grad) return PALSGD_EINVAL;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const size_t n = ctx->n_tensors;
     const size_t gs = elem_size_param(ctx->cfg.precision);
     if (!finite_nonneg(lr_t) || !finite_nonneg(eta_t)) return PALSGD_EINVAL;
     const uint32_t K = ctx->cfg.K;
     for (uint32_t k = 0; k < K; ++k) {                       // a pulling worker's pointers are not looked at
-        if (draw_pull(ctx->cfg.seed, ctx->t, k, ctx->thr)) continue;
+        if (draw_pull(ctx->cfg.seed, ctx->t, ctx->k0 + k, ctx->thr)) continue;
         for (size_t j = 0; j < n; ++j)
             if (!h_grad[(size_t)k * n + j] && ctx->numel[j] > 0) return PALSGD_EINVAL;
     }
+    // everything is checked before the first enqueue: the global model is read back only on a sync step
+    const bool will_sync = (ctx->t + 1) % ctx->cfg.H == 0;
+    if (will_sync && h_global)
+        for (size_t j = 0; j < n; ++j)
+            if (!h_global[j] && ctx->numel[j] > 0) return PALSGD_EINVAL;
     // host -> device gradients of worker k; tensors adjacent on both sides travel as one copy.
     // A worker that pulls in this step has no use for a gradient (Algorithm 1 takes one branch or the
     // other), so nothing is transferred for it.
     auto copy_worker = [&](uint32_t k, cudaStream_t cs) -> int {
-        if (draw_pull(ctx->cfg.seed, ctx->t, k, ctx->thr)) return PALSGD_OK;
+        if (draw_pull(ctx->cfg.seed, ctx->t, ctx->k0 + k, ctx->thr)) return PALSGD_OK;
         for (const Segment& sg : ctx->segs) {
             size_t j = sg.first_tensor;
             const size_t end = sg.first_tensor + sg.n_tensors;
@@ -791,7 +878,6 @@ extern "C" int palsgd_step_host(palsgd_ctx* ctx, const void* const* h_grad, doub
             const size_t end = sg.first_tensor + sg.n_tensors;
             while (j < end) {
                 char* dst = reinterpret_cast<char*>(h_global[j]);
-                if (!dst) return PALSGD_EINVAL;
                 size_t bytes = ctx->numel[j] * 4;
                 size_t j2 = j + 1;
                 while (j2 < end && reinterpret_cast<char*>(h_global[j2]) == dst + bytes) {
@@ -813,7 +899,7 @@ extern "C" int palsgd_step_host(palsgd_ctx* ctx, const void* const* h_grad, doub
 extern "C" int palsgd_get_counters(palsgd_ctx* ctx, uint64_t* t, uint64_t* s_k, uint64_t* n_outer,
                                    uint8_t* last_b, void* stream)
 {
-    if (!ctx) return PALSGD_EINVAL;
+    PALSGD_USABLE(ctx);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     DevState hs;
     PALSGD_CUDA(ctx, cudaMemcpyAsync(&hs, ctx->tb.st, sizeof(hs), cudaMemcpyDeviceToHost, s));
@@ -824,14 +910,14 @@ extern "C" int palsgd_get_counters(palsgd_ctx* ctx, uint64_t* t, uint64_t* s_k, 
         if (s_k) s_k[k] = hs.s[k];
         if (last_b) last_b[k] = hs.last_b[k];
     }
-    if (hs.error != 0) return PALSGD_ETIMEOUT;
     return hs.t == ctx->t ? PALSGD_OK : PALSGD_ESTATE;
 }
 
 extern "C" int palsgd_set_counters(palsgd_ctx* ctx, uint64_t t, const uint64_t* s_k, uint64_t n_outer,
                                    void* stream)
 {
-    if (!ctx || !s_k) return PALSGD_EINVAL;
+    PALSGD_USABLE(ctx);
+    if (!s_k) return PALSGD_EINVAL;
     for (uint32_t k = 0; k < ctx->cfg.K; ++k)
         if (s_k[k] > t) return PALSGD_EINVAL;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -891,7 +977,7 @@ extern "C" int palsgd_set_grad_clip(palsgd_ctx* ctx, double max_norm)
 
 extern "C" int palsgd_get_grad_norms(palsgd_ctx* ctx, double* sumsq, float* clip, void* stream)
 {
-    if (!ctx) return PALSGD_EINVAL;
+    PALSGD_USABLE(ctx);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     DevState hs;
     PALSGD_CUDA(ctx, cudaMemcpyAsync(&hs, ctx->tb.st, sizeof(hs), cudaMemcpyDeviceToHost, s));
@@ -910,19 +996,30 @@ extern "C" int palsgd_get_launch_count(palsgd_ctx* ctx, uint64_t* n_launches)
     return PALSGD_OK;
 }
 
+extern "C" int palsgd_get_layout(palsgd_ctx* ctx, uint64_t* n_segments, uint64_t* n_chunks, uint32_t* chunk_elems)
+{
+    if (!ctx) return PALSGD_EINVAL;
+    if (n_segments) *n_segments = ctx->segs.size();
+    if (n_chunks) *n_chunks = ctx->tb.n_chunks;
+    if (chunk_elems) *chunk_elems = ctx->chunk_elems;
+    return PALSGD_OK;
+}
+
 extern "C" int palsgd_set_tuning(palsgd_ctx* ctx, int knob, int64_t value)
 {
     if (!ctx || value < 0 || value > 0x7FFFFFFF) return PALSGD_EINVAL;
     switch (knob) {
         case PALSGD_TUNE_INNER_GRID_CAP: ctx->grid_cap_inner = (int)value; return PALSGD_OK;
         case PALSGD_TUNE_OUTER_GRID_CAP: ctx->grid_cap_outer = (int)value; return PALSGD_OK;
-        case PALSGD_TUNE_INNER_VARIANT:  ctx->inner_variant = (int)value; return PALSGD_OK;
-        case PALSGD_TUNE_PIPE_STAGES:    ctx->pipe_stages = (int)value; return PALSGD_OK;
-        case PALSGD_TUNE_CHUNK_MAJOR:    ctx->chunk_major = value != 0; return PALSGD_OK;
-        case PALSGD_TUNE_OUTER_SUB_ELEMS:
-            if (value < 1024 || value % 1024 != 0) return PALSGD_EINVAL;
-            ctx->outer_sub_elems = (uint32_t)value;
+        case PALSGD_TUNE_INNER_VARIANT:
+            if (value != 0 && value != 18) return PALSGD_EINVAL;
+            ctx->inner_variant = (int)value;
             return PALSGD_OK;
+        case PALSGD_TUNE_OUTER_SUB_ELEMS:
+            if (value < 1024 || value % 1024 != 0 || value > (1 << 20)) return PALSGD_EINVAL;
+            if (ctx->failed) return PALSGD_ESTATE;
+            ctx->outer_sub_elems = (uint32_t)value;
+            return upload_items(ctx, cut_segments(ctx->segs, ctx->outer_sub_elems), &ctx->d_oitems, &ctx->n_oitems);
         case PALSGD_TUNE_OUTER_DYNAMIC:
             if (value > 32) return PALSGD_EINVAL;
             ctx->outer_dynamic = (int)value;
@@ -936,9 +1033,10 @@ extern "C" int palsgd_set_tuning(palsgd_ctx* ctx, int knob, int64_t value)
             ctx->ddp_variant = (int)value;
             return PALSGD_OK;
         case PALSGD_TUNE_DDP_SUB_ELEMS:
-            if (value < 1024 || value % 1024 != 0) return PALSGD_EINVAL;
+            if (value < 1024 || value % 1024 != 0 || value > (1 << 20)) return PALSGD_EINVAL;
+            if (ctx->failed) return PALSGD_ESTATE;
             ctx->ddp_sub_elems = (uint32_t)value;
-            return PALSGD_OK;
+            return upload_items(ctx, cut_segments(ctx->segs, ctx->ddp_sub_elems), &ctx->d_ditems, &ctx->n_ditems);
         default: return PALSGD_EINVAL;
     }
 }
@@ -947,7 +1045,7 @@ extern "C" int palsgd_set_tuning(palsgd_ctx* ctx, int knob, int64_t value)
 
 extern "C" int palsgd_decision(uint64_t seed, uint64_t t, uint32_t k, double p)
 {
-    if (!(p >= 0.0 && p <= 1.0) || k >= PALSGD_MAX_WORKERS) return PALSGD_EINVAL;
+    if (!(p >= 0.0 && p <= 1.0)) return PALSGD_EINVAL;
     return draw_pull(seed, t, k, threshold_of(p)) ? 1 : 0;
 }
 
@@ -961,7 +1059,6 @@ extern "C" const char* palsgd_strerror(int status)
         case PALSGD_ESTATE: return "call not valid in this state";
         case PALSGD_ENOMEM: return "out of memory";
         case PALSGD_EUNSUPPORTED: return "unsupported combination";
-        case PALSGD_ETIMEOUT: return "a bounded device-side wait expired";
         case PALSGD_ETOOBIG: return "tensor list exceeds the fixed scratch of the no-allocation entry point";
         default: return "unknown status";
     }
@@ -979,6 +1076,8 @@ extern "C" void palsgd_destroy(palsgd_ctx* ctx)
     for (cudaEvent_t e : ctx->copy_done) if (e) cudaEventDestroy(e);
     if (ctx->copy_may_start) cudaEventDestroy(ctx->copy_may_start);
     if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
+    if (ctx->d_oitems) cudaFree(ctx->d_oitems);
+    if (ctx->d_ditems) cudaFree(ctx->d_ditems);
     if (ctx->d_blob) cudaFree(ctx->d_blob);
     delete ctx;
 }

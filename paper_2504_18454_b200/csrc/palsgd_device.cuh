@@ -10,16 +10,16 @@ constexpr uint32_t kMaxWorkers  = 64;      // K <= 64 (worker masks are 64-bit)
 constexpr uint32_t kThreads     = 256;     // threads per CTA of every kernel here
 constexpr uint32_t kChunkElems  = 8192;    // default elements per chunk-table entry = one work item of the
                                            // inner kernel (large: amortises the per-CTA prologue and tick)
-constexpr uint32_t kStageElems  = 4096;    // stage size of the shared-memory-ring kernels
-constexpr uint32_t kOuterSubElems = 1024;  // default work item of the outer kernel for K >= 8: a slice of a
-                                           // chunk (small: K+2 streams per element need many CTAs in flight)
-constexpr uint32_t kDdpSubElems = 1024;    // default work item of the DDP warm-up kernel in fp32 mode (measured
-                                           // with the persistent grid; 4096 in bf16 mode)
+constexpr uint32_t kOuterSubElems = 1024;  // default work item of the outer kernel for K >= 8 (small: K+2
+                                           // streams per element need many CTAs in flight)
+constexpr uint32_t kDdpSubElems = 1024;    // default work item of the DDP warm-up kernel in fp32 mode
 constexpr uint32_t kSegVecFlag  = 0x80000000u;   // Chunk::seg bit: 16-byte vector path allowed
 
 // One work unit of the multi-tensor launch: `len` consecutive elements of
 // segment `seg` starting at element `off`.  A segment is a maximal run of the
-// caller's tensors that are adjacent in memory in every buffer.
+// caller's tensors that are adjacent in memory in every buffer.  The same
+// record serves the chunk table of the inner kernel and the (finer) item
+// tables of the outer-sync and DDP kernels.
 struct Chunk {
     uint64_t off;
     uint32_t len;
@@ -36,7 +36,7 @@ struct DevState {
     double             pow2[kMaxWorkers];    // beta2^s_k
     unsigned int       queue;                // next work item of a launch that hands items out dynamically
     unsigned int       done;                 // CTAs that finished the current inner launch
-    unsigned int       error;                // 0, or the code of a bounded wait that expired
+    unsigned int       pad0_;
     unsigned char      last_b[kMaxWorkers];  // decisions of the latest inner step
     // global-norm gradient clipping (written by the norm kernel, read by the step kernels)
     unsigned int       done_norm;            // CTAs that finished the current norm launch
@@ -51,9 +51,7 @@ struct Tables {
     uint32_t            n_chunks;
     uint32_t            n_seg;
     uint32_t            K;
-    uint32_t            n_full;     // the first n_full chunks are full-size and 16-byte aligned
     uint32_t            chunk_elems; // elements of a full chunk
-    uint32_t            pad_;
     float* const*       xf;         // fp32 model of slot k: params (FP32) or master (BF16_MASTER)
     __nv_bfloat16* const* xw;       // bf16 working params (BF16_MASTER) else nullptr
     const void* const*  grad;       // float or bf16 gradients
@@ -62,6 +60,7 @@ struct Tables {
     float* const*       global;     // [n_seg]
     float* const*       outer_mom;  // [n_seg]
     float* const*       outer_v;    // [n_seg] second outer moment (AdamW as OuterOPT) or nullptr
+    const uint64_t*     exch_off;   // [n_seg] element offset of the segment inside the exchange buffer
     DevState*           st;
     double2*            norm_part;  // [n_chunks * K] per-work-item partial sums of squares (hi, lo)
 };
@@ -75,10 +74,10 @@ struct InnerArgs {
     float    beta_pull;    // fl32(alpha_t * eta_t / p)
     float    b1, b2, omb1, omb2, eps, decay;   // AdamW scalars, each rounded once from binary64
     float    mu, wd;       // momentum SGD scalars
-    uint32_t chunk_major;  // 0: worker index fastest over work items; 1: chunk index fastest
     uint32_t clip_on;      // 1: scale worker k's gradient by DevState::clip[k]
     uint32_t k_begin;      // this launch covers workers k_begin .. k_begin + k_count - 1 (default: all K)
     uint32_t k_count;
+    uint32_t k0;           // the decision stream's index of local worker 0 (workers spread over several contexts)
     uint32_t tick;         // 1: the last CTA advances the device counters (the launch that completes a step)
     uint32_t dynamic;      // 1: a persistent grid takes work items from DevState::queue (needs tick = 1)
 };
@@ -91,12 +90,16 @@ struct PullArgs {
 
 struct OuterArgs {
     Tables tb;
+    const Chunk* items;    // work items: pieces of at most sub_elems elements of a segment
+    uint32_t n_items;
     float  mu, lr, Kf;
     int    nesterov;
     float  ob1, ob2, oomb1, oomb2, obc1, obc2, odecay, oeps;   // AdamW as OuterOPT (step n_outer + 1)
-    uint32_t sub_elems;    // elements per work item (a multiple of 4 * kThreads)
-    uint32_t parts;        // work items per chunk = ceil(chunk_elems / sub_elems)
+    uint32_t sub_elems;    // largest work item (a multiple of 4 * kThreads): size of a stage array
+    uint32_t n_stage;      // stage buffers in dynamic shared memory: 2 for a persistent grid, else 1
     uint32_t dynamic;      // 1: a persistent grid takes work items from DevState::queue
+    const float* sum_in;   // SUMIN kernels: the exchange buffer holding the sum over ALL workers' models
+    float*       sum_out;  // partial-sum kernel: the exchange buffer that receives the local workers' sum
 };
 
 // DDP warm-up step: averaged gradient, one optimizer step taken on worker 0's state, written to all.
@@ -107,8 +110,10 @@ struct DdpArgs {
     float    b1, b2, omb1, omb2, eps, decay;
     float    mu, wd;
     float    Kf;
-    uint32_t sub_elems;    // elements per work item (a multiple of 4 * kThreads)
-    uint32_t parts;        // work items per chunk
+    const Chunk* items;    // work items: pieces of at most sub_elems elements of a segment
+    uint32_t n_items;
+    uint32_t sub_elems;    // largest work item (a multiple of 4 * kThreads): size of a stage array
+    uint32_t n_stage;      // stage buffers in dynamic shared memory: 2 for a persistent grid, else 1
     uint32_t clip_on;      // 1: scale the averaged gradient by DevState::clip[0]
     uint32_t dynamic;      // 1: a persistent grid takes work items from DevState::queue
 };
@@ -120,6 +125,7 @@ struct NormArgs {
     uint64_t thr;          // decision threshold: workers that pull this step are skipped
     double   max_norm;     // clip threshold
     float    Kf;
+    uint32_t k0;           // the decision stream's index of local worker 0
     uint32_t ddp;          // 0: per-worker norms (Algorithm 1 phase); 1: norm of the averaged gradient
     uint32_t group;        // consecutive chunks per work item (a function of the problem size only)
 };

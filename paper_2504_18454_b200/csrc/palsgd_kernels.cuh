@@ -160,62 +160,6 @@ __device__ __forceinline__ void pull_chunk_f32(uint32_t tid, float* __restrict__
 }
 
 
-// ---- fp32 bodies with two ADJACENT 128-bit accesses per stream and thread (8 elements, whole
-// 32-byte sectors per thread).  Selected with U = -1 in grad_item / pull_item.
-template <int INNER, int NT>
-__device__ __forceinline__ void grad_chunk_f32_pair(uint32_t tid, const float* __restrict__ g, float* __restrict__ x,
-                                                    float* __restrict__ m, float* __restrict__ v, uint32_t len,
-                                                    const AdamScalars& as, const SgdScalars& ss)
-{
-    const uint32_t n8 = len >> 3;
-    const float4* g4 = reinterpret_cast<const float4*>(g);
-    float4* x4 = reinterpret_cast<float4*>(x);
-    float4* m4 = reinterpret_cast<float4*>(m);
-    float4* v4 = reinterpret_cast<float4*>(v);
-    for (uint32_t i = tid; i < n8; i += NT) {
-        float4 G[2], X[2], M[2], V[2];
-#pragma unroll
-        for (int c2 = 0; c2 < 2; ++c2) {
-            G[c2] = ld_stream(g4 + 2 * i + c2); X[c2] = ld_stream(x4 + 2 * i + c2);
-            M[c2] = ld_stream(m4 + 2 * i + c2);
-            if (INNER == 0) V[c2] = ld_stream(v4 + 2 * i + c2);
-        }
-#pragma unroll
-        for (int c2 = 0; c2 < 2; ++c2) {
-            if (INNER == 0) { PALSGD_FOR4(adamw_elem(compv(G[c2], c), comp(X[c2], c), comp(M[c2], c), comp(V[c2], c), as)) }
-            else            { PALSGD_FOR4(sgdm_elem(compv(G[c2], c), comp(X[c2], c), comp(M[c2], c), ss)) }
-            st_stream(x4 + 2 * i + c2, X[c2]); st_stream(m4 + 2 * i + c2, M[c2]);
-            if (INNER == 0) st_stream(v4 + 2 * i + c2, V[c2]);
-        }
-    }
-    for (uint32_t i = (n8 << 3) + tid; i < len; i += NT) {
-        float xi = x[i], mi = m[i];
-        if (INNER == 0) { float vi = v[i]; adamw_elem(g[i], xi, mi, vi, as); v[i] = vi; }
-        else            { sgdm_elem(g[i], xi, mi, ss); }
-        x[i] = xi; m[i] = mi;
-    }
-}
-
-template <int NT>
-__device__ __forceinline__ void pull_chunk_f32_pair(uint32_t tid, float* __restrict__ x, const float* __restrict__ xg,
-                                                    uint32_t len, float beta)
-{
-    const uint32_t n8 = len >> 3;
-    float4* x4 = reinterpret_cast<float4*>(x);
-    const float4* q4 = reinterpret_cast<const float4*>(xg);
-    for (uint32_t i = tid; i < n8; i += NT) {
-        float4 X[2], Q[2];
-#pragma unroll
-        for (int c2 = 0; c2 < 2; ++c2) { X[c2] = ld_stream(x4 + 2 * i + c2); Q[c2] = __ldg(q4 + 2 * i + c2); }
-#pragma unroll
-        for (int c2 = 0; c2 < 2; ++c2) {
-            PALSGD_FOR4(comp(X[c2], c) = pull_elem(compv(X[c2], c), compv(Q[c2], c), beta))
-            st_stream(x4 + 2 * i + c2, X[c2]);
-        }
-    }
-    for (uint32_t i = (n8 << 3) + tid; i < len; i += NT) x[i] = pull_elem(x[i], xg[i], beta);
-}
-
 // ---------------------------------------------------------------- bf16 + fp32-master chunk bodies
 // Groups of 8 elements: one 128-bit load of bf16 gradients, two per fp32 stream.
 
@@ -348,8 +292,7 @@ __device__ __forceinline__ void pull_chunk_bf16(uint32_t tid, __nv_bfloat16* __r
 }
 
 
-// ---- bf16 mode with 4-element units (64-bit accesses to the bf16 streams): fewer registers
-// per thread, so more CTAs are resident per SM.  Selected with U = 0 in grad_item / pull_item.
+// 4-element groups of bf16 values (64-bit accesses), used where a thread owns one 128-bit fp32 position
 __device__ __forceinline__ void unpack4(const uint2& h, float (&f)[4])
 {
     f[0] = bf16_bits_to_f32(h.x & 0xFFFFu); f[1] = __uint_as_float(h.x & 0xFFFF0000u);
@@ -358,57 +301,6 @@ __device__ __forceinline__ void unpack4(const uint2& h, float (&f)[4])
 __device__ __forceinline__ uint2 pack4(const float4& a)
 {
     return make_uint2(pack_bf16x2(a.x, a.y), pack_bf16x2(a.z, a.w));
-}
-
-template <int INNER, int NT>
-__device__ __forceinline__ void grad_chunk_bf16_u4(uint32_t tid, const __nv_bfloat16* __restrict__ g,
-                                                   __nv_bfloat16* __restrict__ w, float* __restrict__ x,
-                                                   float* __restrict__ m, float* __restrict__ v, uint32_t len,
-                                                   const AdamScalars& as, const SgdScalars& ss)
-{
-    const uint32_t n4 = len >> 2;
-    const uint2* g4 = reinterpret_cast<const uint2*>(g);
-    uint2* w4 = reinterpret_cast<uint2*>(w);
-    float4* x4 = reinterpret_cast<float4*>(x);
-    float4* m4 = reinterpret_cast<float4*>(m);
-    float4* v4 = reinterpret_cast<float4*>(v);
-    for (uint32_t i = tid; i < n4; i += NT) {
-        const uint2 G = ld_stream(g4 + i);
-        float4 X = ld_stream(x4 + i), M = ld_stream(m4 + i), V;
-        if (INNER == 0) V = ld_stream(v4 + i);
-        float gf[4]; unpack4(G, gf);
-        if (INNER == 0) { PALSGD_FOR4(adamw_elem(gf[c], comp(X, c), comp(M, c), comp(V, c), as)) }
-        else            { PALSGD_FOR4(sgdm_elem(gf[c], comp(X, c), comp(M, c), ss)) }
-        st_stream(x4 + i, X); st_stream(m4 + i, M);
-        if (INNER == 0) st_stream(v4 + i, V);
-        st_stream(w4 + i, pack4(X));
-    }
-    const uint32_t i = (n4 << 2) + tid;
-    if (i < len) {
-        float xi = x[i], mi = m[i];
-        if (INNER == 0) { float vi = v[i]; adamw_elem(__bfloat162float(g[i]), xi, mi, vi, as); v[i] = vi; }
-        else            { sgdm_elem(__bfloat162float(g[i]), xi, mi, ss); }
-        x[i] = xi; m[i] = mi; w[i] = __float2bfloat16_rn(xi);
-    }
-}
-
-template <int NT>
-__device__ __forceinline__ void pull_chunk_bf16_u4(uint32_t tid, __nv_bfloat16* __restrict__ w, float* __restrict__ x,
-                                                   const float* __restrict__ xg, uint32_t len, float beta)
-{
-    const uint32_t n4 = len >> 2;
-    uint2* w4 = reinterpret_cast<uint2*>(w);
-    float4* x4 = reinterpret_cast<float4*>(x);
-    const float4* q4 = reinterpret_cast<const float4*>(xg);
-    for (uint32_t i = tid; i < n4; i += NT) {
-        float4 X = ld_stream(x4 + i);
-        const float4 Q = __ldg(q4 + i);
-        PALSGD_FOR4(comp(X, c) = pull_elem(compv(X, c), compv(Q, c), beta))
-        st_stream(x4 + i, X);
-        st_stream(w4 + i, pack4(X));
-    }
-    const uint32_t i = (n4 << 2) + tid;
-    if (i < len) { const float xi = pull_elem(x[i], xg[i], beta); x[i] = xi; w[i] = __float2bfloat16_rn(xi); }
 }
 
 // ---------------------------------------------------------------- scalar bodies (unaligned segments)
@@ -449,10 +341,8 @@ __device__ __forceinline__ void pull_item(uint32_t tid, const Tables& tb, uint32
     const float* xg = tb.global[seg] + ch.off;
     __nv_bfloat16* w = PREC ? tb.xw[pi] + ch.off : nullptr;
     if (ch.seg & kSegVecFlag) {
-        if (PREC && U == 0) pull_chunk_bf16_u4<NT>(tid, w, x, xg, ch.len, beta);
-        else if (PREC) pull_chunk_bf16<(U > 0 ? U : 1), NT>(tid, w, x, xg, ch.len, beta);
-        else if (U == -1) pull_chunk_f32_pair<NT>(tid, x, xg, ch.len, beta);
-        else      pull_chunk_f32<(U > 0 ? U : 1), NT>(tid, x, xg, ch.len, beta);
+        if (PREC) pull_chunk_bf16<U, NT>(tid, w, x, xg, ch.len, beta);
+        else      pull_chunk_f32<U, NT>(tid, x, xg, ch.len, beta);
     } else {
         pull_chunk_scalar<PREC, NT>(tid, w, x, xg, ch.len, beta);
     }
@@ -471,18 +361,16 @@ __device__ __forceinline__ void grad_item(uint32_t tid, const Tables& tb, uint32
         const __nv_bfloat16* g = static_cast<const __nv_bfloat16*>(tb.grad[pi]) + ch.off;
         __nv_bfloat16* w = tb.xw[pi] + ch.off;
         if (ch.seg & kSegVecFlag) {
-            if (U == 0)          grad_chunk_bf16_u4<INNER, NT>(tid, g, w, x, m, v, ch.len, as, ss);
-            else if (INNER == 0) adamw_chunk_bf16<(U > 0 ? U : 1), NT>(tid, g, w, x, m, v, ch.len, as);
-            else                 sgdm_chunk_bf16<(U > 0 ? U : 1), NT>(tid, g, w, x, m, ch.len, ss);
+            if (INNER == 0) adamw_chunk_bf16<U, NT>(tid, g, w, x, m, v, ch.len, as);
+            else            sgdm_chunk_bf16<U, NT>(tid, g, w, x, m, ch.len, ss);
         } else {
             grad_chunk_scalar<INNER, 1, NT>(tid, g, w, x, m, v, ch.len, as, ss);
         }
     } else {
         const float* g = static_cast<const float*>(tb.grad[pi]) + ch.off;
         if (ch.seg & kSegVecFlag) {
-            if (U == -1)         grad_chunk_f32_pair<INNER, NT>(tid, g, x, m, v, ch.len, as, ss);
-            else if (INNER == 0) adamw_chunk_f32<(U > 0 ? U : 1), NT>(tid, g, x, m, v, ch.len, as);
-            else                 sgdm_chunk_f32<(U > 0 ? U : 1), NT>(tid, g, x, m, ch.len, ss);
+            if (INNER == 0) adamw_chunk_f32<U, NT>(tid, g, x, m, v, ch.len, as);
+            else            sgdm_chunk_f32<U, NT>(tid, g, x, m, ch.len, ss);
         } else {
             grad_chunk_scalar<INNER, 0, NT>(tid, g, nullptr, x, m, v, ch.len, as, ss);
         }
@@ -509,7 +397,7 @@ palsgd_inner_kernel(const __grid_constant__ InnerArgs a)
 
     if (threadIdx.x < K) {
         const uint32_t k = threadIdx.x;
-        const bool pull = draw_pull(a.seed, t, k, a.thr);
+        const bool pull = draw_pull(a.seed, t, a.k0 + k, a.thr);
         s_pull[k] = pull;
         s_clip[k] = a.clip_on ? st->clip[k] : 1.f;
         if (INNER == 0 && !pull) {                       // bias corrections for gradient step s_k + 1
@@ -533,8 +421,8 @@ palsgd_inner_kernel(const __grid_constant__ InnerArgs a)
         item = s_item;
     }
     while (item < n_items) {
-        const uint32_t k = a.k_begin + (uint32_t)(a.chunk_major ? item / tb.n_chunks : item % Kc);
-        const Chunk ch = tb.chunks[a.chunk_major ? item % tb.n_chunks : item / Kc];
+        const uint32_t k = a.k_begin + (uint32_t)(item % Kc);
+        const Chunk ch = tb.chunks[item / Kc];
         if (s_pull[k]) {
             pull_item<PREC, U, kThreads>(threadIdx.x, tb, k, ch, a.beta_pull);
         } else {
@@ -589,23 +477,41 @@ palsgd_pull_kernel(const __grid_constant__ PullArgs a)
 }
 
 // ---------------------------------------------------------------- work distribution
-// Next work item of a CTA: strided by the grid, or (dynamic) drawn from a counter in device memory by
-// a persistent grid.  Called by all threads of the CTA; s_item is a shared-memory word of the caller.
-__device__ __forceinline__ uint64_t first_item(uint32_t dynamic, DevState* st, unsigned int* s_item)
-{
-    if (!dynamic) return blockIdx.x;
-    if (threadIdx.x == 0) *s_item = atomicAdd(&st->queue, 1u);
-    __syncthreads();
-    return *s_item;
-}
-__device__ __forceinline__ uint64_t next_item(uint64_t cur, uint32_t dynamic, DevState* st, unsigned int* s_item)
-{
-    if (!dynamic) return cur + gridDim.x;
-    __syncthreads();                                           // everyone has read *s_item
-    if (threadIdx.x == 0) *s_item = atomicAdd(&st->queue, 1u);
-    __syncthreads();
-    return *s_item;
-}
+// The outer-sync and DDP kernels walk an item table either strided by the grid or (dynamic) as a
+// persistent grid that draws item indices from a counter in device memory.  The index of the NEXT
+// item is requested once the current one has been computed (the atomic's round trip hides behind the
+// fan-out of its results; requested earlier, in the middle of the load loop, the atomic kept the
+// compiler from overlapping the loop's loads and cost the DDP kernel 15 %) and handed to the CTA
+// through a two-slot mailbox in shared memory: slot (n+1)&1 is written during item n and read after
+// the barrier that closes it, so one barrier per item orders everything.
+struct ItemWalk {
+    unsigned int* slots;        // two words of shared memory
+    uint32_t      dynamic;
+    DevState*     st;
+    uint32_t      n;            // items done by this CTA
+    unsigned int  pending;      // thread 0: the index requested for the next item
+
+    __device__ __forceinline__ uint32_t first()
+    {
+        n = 0;
+        if (threadIdx.x == 0) slots[0] = dynamic ? atomicAdd(&st->queue, 1u) : blockIdx.x;
+        __syncthreads();
+        return slots[0];
+    }
+    // call once the current item has been computed
+    __device__ __forceinline__ void request_next(uint32_t cur)
+    {
+        if (threadIdx.x == 0) pending = dynamic ? atomicAdd(&st->queue, 1u) : cur + gridDim.x;
+    }
+    // call at the end of the item; contains the item's closing barrier
+    __device__ __forceinline__ uint32_t next()
+    {
+        ++n;
+        if (threadIdx.x == 0) slots[n & 1] = pending;
+        __syncthreads();
+        return slots[n & 1];
+    }
+};
 // After the loop of a dynamic launch: the last CTA to finish rewinds the queue for the next launch.
 __device__ __forceinline__ void rewind_queue(DevState* st)
 {
@@ -621,17 +527,20 @@ __device__ __forceinline__ void rewind_queue(DevState* st)
 // One result written to K slots: the CTA stages it in shared memory once and a bulk
 // asynchronous copy per slot and stream (cp.async.bulk shared -> global; this GPU's own
 // memory, no multicast) carries it out, instead of K x 128-bit stores per thread.
+// A persistent CTA alternates between two stage buffers: the copies of item n drain while
+// item n+1 is loaded, computed and staged in the other buffer.  Bulk groups are per thread:
+// every issuing thread commits exactly one group per item (an empty one if it has nothing to
+// copy), so "all but the latest group have been read" means "the buffer of two items ago is free".
 __device__ __forceinline__ void bulk_store(void* dst_gmem, const void* src_smem, uint32_t bytes)
 {
     asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
                  ::"l"(__cvta_generic_to_global(dst_gmem)), "r"((uint32_t)__cvta_generic_to_shared(src_smem)), "r"(bytes)
                  : "memory");
 }
-__device__ __forceinline__ void bulk_store_commit_and_wait_read()
-{
-    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-    asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");     // shared memory may be reused after this
-}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// shared memory of all groups but the latest `Pending` ones may be reused after this
+template <int Pending>
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(Pending) : "memory"); }
 // generic-proxy writes to shared memory become visible to the asynchronous proxy
 __device__ __forceinline__ void fence_async_shared() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
@@ -660,33 +569,36 @@ __device__ __forceinline__ float outer_elem_adamw(float sum, float Kf, float xg,
 }
 
 // OOPT: 0 = SGD with (Nesterov) momentum, 1 = AdamW (one more state stream).
-// BCAST = 1: the new global model of a work item (and its bf16 copy) is staged in dynamic shared
-// memory (4 + 2 bytes per element, sub_elems elements) and written to the K slots by bulk
-// asynchronous stores; 16-byte-aligned segments only, the rest takes the register path.
-template <int PREC, int OOPT, int BCAST>
-__global__ void __launch_bounds__(kThreads)
+// BCAST = 1: the new global model of a work item (with u and the bf16 copy) is staged in dynamic
+// shared memory (8 (+4) (+2) bytes per element, sub_elems elements per buffer) and written to x_g,
+// u and the K slots by bulk asynchronous stores; 16-byte-aligned pieces only, the rest takes the
+// register path.
+// SUMIN = 1: the sum over the workers is not formed here but read from the exchange buffer (it was
+// formed by palsgd_outer_partial_kernel on every GPU and all-reduced), and Kf is the number of workers
+// of the whole job; this launch then finishes the synchronisation for the local slots.
+template <int PREC, int OOPT, int BCAST, int SUMIN = 0>
+__global__ void __launch_bounds__(kThreads, (BCAST && !OOPT) ? 4 : 1)      // 64 registers: 4 CTAs per SM
 palsgd_outer_kernel(const __grid_constant__ OuterArgs a)
 {
     extern __shared__ __align__(128) unsigned char outer_stage[];
     const AdamScalars os{a.ob1, a.ob2, a.oomb1, a.oomb2, a.obc1, a.obc2, a.odecay, a.lr, a.oeps};
     __shared__ float* s_x[kMaxWorkers];
     __shared__ __nv_bfloat16* s_w[kMaxWorkers];
+    __shared__ unsigned int s_slots[2];
     const Tables& tb = a.tb;
     const uint32_t K = tb.K;
     constexpr int B = 8;                                   // slot loads issued together
+    const uint32_t stage_bytes = a.sub_elems * (8u + (OOPT ? 4u : 0u) + (PREC ? 2u : 0u));
+    const bool issuer = BCAST && threadIdx.x <= K;         // thread k < K: slot k's copies; thread K: x_g and u
+    const uint32_t Ksum = SUMIN ? 0u : K;                  // slots summed here (none when the sum comes in ready-made)
 
-    __shared__ unsigned int s_item;
-    const uint64_t n_items = (uint64_t)tb.n_chunks * a.parts;
-    for (uint64_t item = first_item(a.dynamic, tb.st, &s_item); item < n_items;
-         item = next_item(item, a.dynamic, tb.st, &s_item)) {
-        Chunk ch = tb.chunks[item / a.parts];
-        const uint32_t begin = (uint32_t)(item % a.parts) * a.sub_elems;      // this item's slice of the chunk
-        if (begin >= ch.len) continue;                                        // uniform over the CTA
-        ch.off += begin;
-        ch.len = min(ch.len - begin, a.sub_elems);
+    ItemWalk walk{s_slots, a.dynamic, tb.st, 0, 0};
+    for (uint32_t item = walk.first(); item < a.n_items; item = walk.next()) {
+        const Chunk ch = a.items[item];
         const uint32_t seg = ch.seg & ~kSegVecFlag;
-        __syncthreads();
-        if (threadIdx.x < K) {
+        // the stage buffer about to be refilled was handed to the copy engine two items ago
+        if (issuer) { if (a.n_stage > 1) bulk_wait_read<1>(); else bulk_wait_read<0>(); }
+        if (threadIdx.x < K) {                             // (the previous item's closing barrier protects s_x)
             const size_t pi = (size_t)threadIdx.x * tb.n_seg + seg;
             s_x[threadIdx.x] = tb.xf[pi] + ch.off;
             if (PREC) s_w[threadIdx.x] = tb.xw[pi] + ch.off;
@@ -695,6 +607,10 @@ palsgd_outer_kernel(const __grid_constant__ OuterArgs a)
         float* xg = tb.global[seg] + ch.off;
         float* um = tb.outer_mom[seg] + ch.off;
         float* uv = OOPT ? tb.outer_v[seg] + ch.off : nullptr;
+        const float* sum_src = SUMIN ? a.sum_in + tb.exch_off[seg] + ch.off : nullptr;
+        unsigned char* stage = outer_stage + (BCAST ? (walk.n % a.n_stage) * stage_bytes : 0u);
+        float* sx = reinterpret_cast<float*>(stage);
+        float* su = sx + a.sub_elems;
 
         uint32_t done = 0;
         if (ch.seg & kSegVecFlag) {
@@ -705,7 +621,15 @@ palsgd_outer_kernel(const __grid_constant__ OuterArgs a)
                 float4 Uv = make_float4(0.f, 0.f, 0.f, 0.f);
                 if (OOPT) Uv = __ldcs(reinterpret_cast<const float4*>(uv) + i);
                 float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-                for (uint32_t k0 = 0; k0 < K; k0 += B) {
+                if (SUMIN) {
+                    // the exchange buffer packs the tensors back to back: a piece may sit off 16-byte alignment there
+                    if ((reinterpret_cast<uintptr_t>(sum_src) & 15u) == 0)
+                        acc = __ldcs(reinterpret_cast<const float4*>(sum_src) + i);
+                    else
+                        acc = make_float4(__ldcs(sum_src + 4 * i), __ldcs(sum_src + 4 * i + 1),
+                                          __ldcs(sum_src + 4 * i + 2), __ldcs(sum_src + 4 * i + 3));
+                }
+                for (uint32_t k0 = 0; k0 < Ksum; k0 += B) {
                     float4 R[B];
 #pragma unroll
                     for (int j = 0; j < B; ++j)
@@ -734,8 +658,6 @@ palsgd_outer_kernel(const __grid_constant__ OuterArgs a)
                     // x_g and u have one destination each and are written once the fan-out below has
                     // been fixed (a group of 4 left over by the bf16 16-byte rule is redone by the
                     // scalar loop from unmodified inputs), so they are staged too
-                    float* sx = reinterpret_cast<float*>(outer_stage);
-                    float* su = sx + a.sub_elems;
                     reinterpret_cast<float4*>(sx)[i] = N;
                     reinterpret_cast<float4*>(su)[i] = Um;
                     if (OOPT) reinterpret_cast<float4*>(su + a.sub_elems)[i] = Uv;
@@ -753,30 +675,29 @@ palsgd_outer_kernel(const __grid_constant__ OuterArgs a)
                 }
             }
             done = n4 << 2;
-            if (BCAST) {
-                const uint32_t lenb = PREC ? (done & ~7u) : done;       // whole 16-byte units of every stream
-                fence_async_shared();
-                __syncthreads();
-                if (lenb > 0 && threadIdx.x <= K) {
-                    const float* sx = reinterpret_cast<const float*>(outer_stage);
-                    const float* su = sx + a.sub_elems;
+            if (BCAST) done = PREC ? (done & ~7u) : done;       // whole 16-byte units of every stream
+        }
+        walk.request_next(item);                            // its round trip hides behind the fan-out below
+        if (BCAST) {
+            fence_async_shared();
+            __syncthreads();
+            if (issuer) {
+                if (done > 0) {
                     if (threadIdx.x == K) {
-                        bulk_store(xg, sx, lenb * 4);
-                        bulk_store(um, su, lenb * 4);
-                        if (OOPT) bulk_store(uv, su + a.sub_elems, lenb * 4);
+                        bulk_store(xg, sx, done * 4);
+                        bulk_store(um, su, done * 4);
+                        if (OOPT) bulk_store(uv, su + a.sub_elems, done * 4);
                     } else {
-                        bulk_store(s_x[threadIdx.x], sx, lenb * 4);
-                        if (PREC) bulk_store(s_w[threadIdx.x], su + (OOPT ? 2 : 1) * a.sub_elems, lenb * 2);
+                        bulk_store(s_x[threadIdx.x], sx, done * 4);
+                        if (PREC) bulk_store(s_w[threadIdx.x], su + (OOPT ? 2 : 1) * a.sub_elems, done * 2);
                     }
-                    bulk_store_commit_and_wait_read();
                 }
-                done = lenb;
-                __syncthreads();                             // the stage may be overwritten by the next item
+                bulk_commit();                                  // one group per item, possibly empty
             }
         }
         for (uint32_t i = done + threadIdx.x; i < ch.len; i += kThreads) {
-            float sum = s_x[0][i];
-            for (uint32_t k = 1; k < K; ++k) sum = __fadd_rn(sum, s_x[k][i]);
+            float sum = SUMIN ? sum_src[i] : s_x[0][i];
+            for (uint32_t k = 1; k < Ksum; ++k) sum = __fadd_rn(sum, s_x[k][i]);
             float ui = um[i], xn;
             if (OOPT) { float vi = uv[i]; xn = outer_elem_adamw(sum, a.Kf, xg[i], ui, vi, os); uv[i] = vi; }
             else      { xn = outer_elem(sum, a.Kf, xg[i], ui, a.mu, a.lr, a.nesterov); }
@@ -786,7 +707,60 @@ palsgd_outer_kernel(const __grid_constant__ OuterArgs a)
                         for (uint32_t k = 0; k < K; ++k) s_w[k][i] = h; }
         }
     }
+    if (issuer) bulk_wait_read<0>();                            // shared memory must outlive the copies' reads
     if (a.dynamic) rewind_queue(tb.st);
+}
+
+// ---------------------------------------------------------------- outer sync over several GPUs, first half
+// Algorithm 1's All-Reduce when the K workers are spread over several GPUs: every GPU adds up its
+// local workers' models in ascending local index and leaves the sum in the exchange buffer; the
+// buffers are then summed across GPUs by the caller's collective, and palsgd_outer_kernel<.., SUMIN>
+// divides by the job's worker count and finishes (Eq. (3), Eq. (4), restart of the local slots).
+template <int B = 8>                                       // B: slot loads issued together
+__global__ void __launch_bounds__(kThreads)
+palsgd_outer_partial_kernel(const __grid_constant__ OuterArgs a)
+{
+    __shared__ float* s_x[kMaxWorkers];
+    const Tables& tb = a.tb;
+    const uint32_t K = tb.K;
+    for (uint32_t item = blockIdx.x; item < a.n_items; item += gridDim.x) {
+        const Chunk ch = a.items[item];
+        const uint32_t seg = ch.seg & ~kSegVecFlag;
+        __syncthreads();
+        if (threadIdx.x < K) s_x[threadIdx.x] = tb.xf[(size_t)threadIdx.x * tb.n_seg + seg] + ch.off;
+        __syncthreads();
+        float* out = a.sum_out + tb.exch_off[seg] + ch.off;
+        uint32_t done = 0;
+        if (ch.seg & kSegVecFlag) {
+            const uint32_t n4 = ch.len >> 2;
+            for (uint32_t i = threadIdx.x; i < n4; i += kThreads) {
+                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                for (uint32_t k0 = 0; k0 < K; k0 += B) {
+                    float4 R[B];
+#pragma unroll
+                    for (int j = 0; j < B; ++j)
+                        if (k0 + j < K) R[j] = __ldcs(reinterpret_cast<const float4*>(s_x[k0 + j]) + i);
+#pragma unroll
+                    for (int j = 0; j < B; ++j)
+                        if (k0 + j < K) {
+                            if (k0 + j == 0) acc = R[j];
+                            else { acc.x = __fadd_rn(acc.x, R[j].x); acc.y = __fadd_rn(acc.y, R[j].y);
+                                   acc.z = __fadd_rn(acc.z, R[j].z); acc.w = __fadd_rn(acc.w, R[j].w); }
+                        }
+                }
+                // (read again soon by the collective: default cache policy; the exchange buffer packs the
+                //  tensors back to back, so a piece may sit off 16-byte alignment there)
+                if ((reinterpret_cast<uintptr_t>(out) & 15u) == 0) reinterpret_cast<float4*>(out)[i] = acc;
+                else { out[4 * i] = acc.x; out[4 * i + 1] = acc.y; out[4 * i + 2] = acc.z; out[4 * i + 3] = acc.w; }
+            }
+            done = n4 << 2;
+        }
+        for (uint32_t i = done + threadIdx.x; i < ch.len; i += kThreads) {
+            float sum = s_x[0][i];
+            for (uint32_t k = 1; k < K; ++k) sum = __fadd_rn(sum, s_x[k][i]);
+            out[i] = sum;
+        }
+    }
 }
 
 // ---------------------------------------------------------------- DDP warm-up step
@@ -794,12 +768,11 @@ palsgd_outer_kernel(const __grid_constant__ OuterArgs a)
 // gradients are summed in ascending k and divided by K, ONE optimizer step is taken on
 // worker 0's model and state with the plain step size alpha_t, and the result goes to
 // every slot and to the global model copy.  Reads 4K+12 bytes (2K+12 with bf16
-// gradients) and writes 12K+4 (14K+4) per parameter for AdamW: store-dominated, so the
-// work item is a small slice of a chunk, as in the outer kernel.
+// gradients) and writes 12K+4 (14K+4) per parameter for AdamW: store-dominated.
 
 // BCAST = 1: the new x, m, v (and bf16 copy) of a work item are staged in dynamic shared memory
-// ((12 or 8) + 2 bytes per element, sub_elems elements) and written to the K slots and to x_g
-// by bulk asynchronous stores; 16-byte-aligned segments only, the rest takes the register path.
+// ((12 or 8) + 2 bytes per element, sub_elems elements per buffer) and written to the K slots and
+// to x_g by bulk asynchronous stores; 16-byte-aligned pieces only, the rest takes the register path.
 template <int INNER, int PREC, int BCAST>
 __global__ void __launch_bounds__(kThreads)
 palsgd_ddp_kernel(const __grid_constant__ DdpArgs a)
@@ -810,10 +783,13 @@ palsgd_ddp_kernel(const __grid_constant__ DdpArgs a)
     __shared__ float* s_v[kMaxWorkers];
     __shared__ const void* s_g[kMaxWorkers];
     __shared__ __nv_bfloat16* s_w[kMaxWorkers];
+    __shared__ unsigned int s_slots[2];
     const Tables& tb = a.tb;
     const uint32_t K = tb.K;
     DevState* st = tb.st;
     constexpr int B = 8;                                   // gradient loads issued together
+    const uint32_t stage_bytes = a.sub_elems * ((INNER == 0 ? 12u : 8u) + (PREC ? 2u : 0u));
+    const bool issuer = BCAST && threadIdx.x <= K;         // thread k < K: slot k's copies; thread K: x_g
 
     // bias corrections for gradient step s_0 + 1 (all workers share worker 0's count in this phase)
     const unsigned long long t = st->t;
@@ -825,18 +801,12 @@ palsgd_ddp_kernel(const __grid_constant__ DdpArgs a)
     SgdScalars ss{a.mu, a.wd, a.lr};
     if (a.clip_on) { as.clip = st->clip[0]; ss.clip = as.clip; }   // the clip applies to the averaged gradient
 
-    __shared__ unsigned int s_item;
-    const uint64_t n_items = (uint64_t)tb.n_chunks * a.parts;
-    for (uint64_t item = first_item(a.dynamic, st, &s_item); item < n_items;
-         item = next_item(item, a.dynamic, st, &s_item)) {
-        Chunk ch = tb.chunks[item / a.parts];
-        const uint32_t begin = (uint32_t)(item % a.parts) * a.sub_elems;
-        if (begin >= ch.len) continue;                                        // uniform over the CTA
-        ch.off += begin;
-        ch.len = min(ch.len - begin, a.sub_elems);
+    ItemWalk walk{s_slots, a.dynamic, st, 0, 0};
+    for (uint32_t item = walk.first(); item < a.n_items; item = walk.next()) {
+        const Chunk ch = a.items[item];
         const uint32_t seg = ch.seg & ~kSegVecFlag;
-        __syncthreads();
-        if (threadIdx.x < K) {
+        if (issuer) { if (a.n_stage > 1) bulk_wait_read<1>(); else bulk_wait_read<0>(); }
+        if (threadIdx.x < K) {                             // (the previous item's closing barrier protects these)
             const size_t pi = (size_t)threadIdx.x * tb.n_seg + seg;
             s_x[threadIdx.x] = tb.xf[pi] + ch.off;
             s_m[threadIdx.x] = tb.m[pi] + ch.off;
@@ -847,6 +817,10 @@ palsgd_ddp_kernel(const __grid_constant__ DdpArgs a)
         }
         __syncthreads();
         float* xg = tb.global[seg] + ch.off;
+        unsigned char* stage = ddp_stage + (BCAST ? (walk.n % a.n_stage) * stage_bytes : 0u);
+        float* sx = reinterpret_cast<float*>(stage);
+        float* sm = sx + a.sub_elems;
+        float* sv = sm + a.sub_elems;
 
         uint32_t done = 0;
         if (ch.seg & kSegVecFlag) {
@@ -880,9 +854,6 @@ palsgd_ddp_kernel(const __grid_constant__ DdpArgs a)
                 if (INNER == 0) { PALSGD_FOR4(adamw_elem(compv(G, c), comp(X, c), comp(M, c), comp(V, c), as)) }
                 else            { PALSGD_FOR4(sgdm_elem(compv(G, c), comp(X, c), comp(M, c), ss)) }
                 if (BCAST) {                                // stage; the fan-out follows the loop
-                    float* sx = reinterpret_cast<float*>(ddp_stage);
-                    float* sm = sx + a.sub_elems;
-                    float* sv = sm + a.sub_elems;
                     reinterpret_cast<float4*>(sx)[i] = X;
                     reinterpret_cast<float4*>(sm)[i] = M;
                     if (INNER == 0) reinterpret_cast<float4*>(sv)[i] = V;
@@ -901,29 +872,27 @@ palsgd_ddp_kernel(const __grid_constant__ DdpArgs a)
                 }
             }
             done = n4 << 2;
-            if (BCAST) {
-                // whole 16-byte units only: the bf16 stream needs a multiple of 8 elements; what is left
-                // of an odd group of 4 is redone below by the scalar loop (its inputs are still intact)
-                const uint32_t lenb = PREC ? (done & ~7u) : done;
-                fence_async_shared();
-                __syncthreads();
-                if (lenb > 0 && threadIdx.x <= K) {
-                    const float* sx = reinterpret_cast<const float*>(ddp_stage);
-                    const float* sm = sx + a.sub_elems;
-                    const float* sv = sm + a.sub_elems;
+            // whole 16-byte units only: the bf16 stream needs a multiple of 8 elements; what is left
+            // of an odd group of 4 is redone below by the scalar loop (its inputs are still intact)
+            if (BCAST) done = PREC ? (done & ~7u) : done;
+        }
+        walk.request_next(item);                            // its round trip hides behind the fan-out below
+        if (BCAST) {
+            fence_async_shared();
+            __syncthreads();
+            if (issuer) {
+                if (done > 0) {
                     if (threadIdx.x == K) {
-                        bulk_store(xg, sx, lenb * 4);
+                        bulk_store(xg, sx, done * 4);
                     } else {
                         const uint32_t k = threadIdx.x;
-                        bulk_store(s_x[k], sx, lenb * 4);
-                        bulk_store(s_m[k], sm, lenb * 4);
-                        if (INNER == 0) bulk_store(s_v[k], sv, lenb * 4);
-                        if (PREC) bulk_store(s_w[k], sm + (INNER == 0 ? 2 : 1) * a.sub_elems, lenb * 2);
+                        bulk_store(s_x[k], sx, done * 4);
+                        bulk_store(s_m[k], sm, done * 4);
+                        if (INNER == 0) bulk_store(s_v[k], sv, done * 4);
+                        if (PREC) bulk_store(s_w[k], sm + (INNER == 0 ? 2 : 1) * a.sub_elems, done * 2);
                     }
-                    bulk_store_commit_and_wait_read();
                 }
-                done = lenb;
-                __syncthreads();                             // the stage may be overwritten by the next item
+                bulk_commit();                                  // one group per item, possibly empty
             }
         }
         for (uint32_t i = done + threadIdx.x; i < ch.len; i += kThreads) {
@@ -945,6 +914,7 @@ palsgd_ddp_kernel(const __grid_constant__ DdpArgs a)
             }
         }
     }
+    if (issuer) bulk_wait_read<0>();                            // shared memory must outlive the copies' reads
 
     // ---- counter tick by the last CTA (all state reads above precede the atomic)
     __syncthreads();

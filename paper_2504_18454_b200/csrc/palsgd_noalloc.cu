@@ -31,7 +31,9 @@ std::mutex g_mutex;                            // guards the cache above and the
 
 // Host-side staging of the tables: fixed size, so that a call allocates nothing
 // on the host either.  cudaMemcpyAsync from pageable memory returns once the
-// bytes have been staged, so the buffer is free again when the call returns.
+// bytes have been staged, so the buffer is free again when the call returns;
+// the runtime waits for the work already enqueued on the stream before it
+// stages them, so the call blocks the host that long.
 alignas(256) unsigned char g_stage[PALSGD_NOALLOC_SCRATCH_BYTES];
 
 inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -100,6 +102,12 @@ extern "C" int palsgd_outer_sync_noalloc(uint32_t K, int32_t precision, size_t n
     if (total > PALSGD_NOALLOC_SCRATCH_BYTES) return PALSGD_ETOOBIG;
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // Not capturable: a captured copy node would re-read the shared host staging buffer, and a captured
+    // kernel node would keep this call's table sizes, at every replay -- after later calls have put
+    // other tables there.  A capturing stream is refused before anything is enqueued.
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(s, &cap) != cudaSuccess) { (void)cudaGetLastError(); return PALSGD_ECUDA; }
+    if (cap != cudaStreamCaptureStatusNone) return PALSGD_ESTATE;
     std::lock_guard<std::mutex> lock(g_mutex);
 
     void* d_void = nullptr;
@@ -152,10 +160,11 @@ extern "C" int palsgd_outer_sync_noalloc(uint32_t K, int32_t precision, size_t n
     a.lr = (float)outer_lr;
     a.Kf = (float)K;
     a.nesterov = outer_nesterov;
-    a.sub_elems = kOuterSubElems;
-    a.parts = (kChunkElems + kOuterSubElems - 1) / kOuterSubElems;
-    const uint64_t n_items = (uint64_t)n_chunks * a.parts;
-    const unsigned grid = (unsigned)(n_items > 0x7FFFFFFFull ? 0x7FFFFFFFull : n_items);
+    a.items = a.tb.chunks;                 // one CTA per 8192-element block, 128-bit stores by every thread
+    a.n_items = (uint32_t)n_chunks;
+    a.sub_elems = kChunkElems;
+    a.n_stage = 1;
+    const unsigned grid = (unsigned)(n_chunks > 0x7FFFFFFFull ? 0x7FFFFFFFull : n_chunks);
     if (bf) palsgd_outer_kernel<1, 0, 0><<<grid, kThreads, 0, s>>>(a);
     else    palsgd_outer_kernel<0, 0, 0><<<grid, kThreads, 0, s>>>(a);
     if (cudaGetLastError() != cudaSuccess) return PALSGD_ECUDA;

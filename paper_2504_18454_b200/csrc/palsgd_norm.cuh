@@ -129,6 +129,78 @@ __device__ __forceinline__ void sumsq_chunk(DD (&q)[4], const void* g, uint32_t 
                                 : static_cast<const float*>(g)[i]);
 }
 
+// ---- bf16 gradients: exact sums at two binary64 operations per element
+// The square of a bf16 value has 16 significant bits, so a run of such squares can be summed
+// EXACTLY in plain binary64 as long as all of them sit within about 2^37 of the running sum.
+// Each chain is kept twice, once with every addition rounded down and once rounded up (the
+// product x*x is exact, so fma_rd / fma_ru round the exact x*x + s once): the chain rounded down
+// never exceeds the exact sum and the chain rounded up never falls below it, hence if the two
+// are EQUAL after a stretch of additions, every addition in it was exact and the common value is
+// the exact sum.  The test is made once per chunk and costs nothing per element.  When it fails
+// (an element far smaller than the running sum, or a NaN), the chains go back to their values at
+// the start of the chunk and this thread's elements of the chunk are added in double-double.
+// Zeros, denormals and infinities need no special case (inf = inf keeps the chains equal).
+struct FastSq {
+    double dn[4], up[4];        // four independent chains (element position mod 4), rounded down / up
+    double ok[4];               // their (common) values at the start of the current chunk
+
+    __device__ __forceinline__ void init()
+    {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) { dn[j] = 0.0; up[j] = 0.0; ok[j] = 0.0; }
+    }
+    __device__ __forceinline__ void add(int j, float g)
+    {
+        const double x = (double)g;
+        dn[j] = __fma_rd(x, x, dn[j]);
+        up[j] = __fma_ru(x, x, up[j]);
+    }
+    // true: every addition since the last call was exact (and the chains are kept);
+    // false: the chains have been put back to where they were at that call
+    __device__ __forceinline__ bool settle()
+    {
+        const bool exact = dn[0] == up[0] && dn[1] == up[1] && dn[2] == up[2] && dn[3] == up[3];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            if (exact) ok[j] = dn[j];
+            else { dn[j] = ok[j]; up[j] = ok[j]; }
+        }
+        return exact;
+    }
+};
+
+// One 16-byte-aligned chunk of one bf16 gradient: this thread's groups of 8 into the fast chains, or,
+// if the chains' test fails for this chunk, once more into the double-double accumulator `slow`.
+__device__ __forceinline__ void sumsq_chunk_bf16_fast(FastSq& f, DD& slow, const void* g, uint32_t len)
+{
+    constexpr int U = 4;
+    const uint4* g8 = static_cast<const uint4*>(g);
+    const uint32_t n8 = len >> 3;
+    for (uint32_t base = 0; base < n8; base += kThreads * U) {
+        uint4 R[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const uint32_t i = base + u * kThreads + threadIdx.x;
+            R[u] = i < n8 ? ld_stream(g8 + i) : make_uint4(0u, 0u, 0u, 0u);      // zeros add nothing
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            float v[8]; unpack8(R[u], v);
+#pragma unroll
+            for (int c = 0; c < 8; ++c) f.add(c & 3, v[c]);
+        }
+    }
+    if (!f.settle()) {                                      // rare; the data is still in cache
+        for (uint32_t i = threadIdx.x; i < n8; i += kThreads) {
+            float v[8]; unpack8(__ldg(g8 + i), v);
+#pragma unroll
+            for (int c = 0; c < 8; ++c) dd_square_in(slow, v[c]);
+        }
+    }
+    for (uint32_t i = (n8 << 3) + threadIdx.x; i < len; i += kThreads)
+        dd_square_in(slow, __bfloat162float(static_cast<const __nv_bfloat16*>(g)[i]));
+}
+
 // One launch ahead of a step whose gradients are clipped.  Work items: (chunk, worker) with the
 // worker index fastest (ddp = 0), or chunks (ddp = 1: the norm of the averaged gradient, formed
 // exactly as the DDP step forms it).  Every item leaves a double-double partial in
@@ -148,7 +220,7 @@ palsgd_gradnorm_kernel(const __grid_constant__ NormArgs a)
     const unsigned long long t = st->t;
     const uint32_t Kitems = a.ddp ? 1u : K;
 
-    if (threadIdx.x < K) s_pull[threadIdx.x] = a.ddp ? 0 : draw_pull(a.seed, t, threadIdx.x, a.thr);
+    if (threadIdx.x < K) s_pull[threadIdx.x] = a.ddp ? 0 : draw_pull(a.seed, t, a.k0 + threadIdx.x, a.thr);
     __syncthreads();
 
     // Work item = a.group consecutive chunks of one worker: the per-thread sums run over the whole
@@ -161,7 +233,24 @@ palsgd_gradnorm_kernel(const __grid_constant__ NormArgs a)
         const uint32_t c_begin = (uint32_t)(item / Kitems) * a.group;
         const uint32_t c_end = min(c_begin + a.group, tb.n_chunks);
         DD q[4] = {{0.0, 0.0}, {0.0, 0.0}, {0.0, 0.0}, {0.0, 0.0}};
-        for (uint32_t c = c_begin; c < c_end; ++c) {
+        bool fast_done = false;
+        if (PREC == 1 && !a.ddp) {
+            // bf16 gradients: plain binary64 chains whose exactness is tested chunk by chunk
+            fast_done = true;
+            if (!s_pull[k]) {
+                FastSq f; f.init();
+                for (uint32_t c = c_begin; c < c_end; ++c) {
+                    const Chunk ch = tb.chunks[c];
+                    const uint32_t seg = ch.seg & ~kSegVecFlag;
+                    const char* g = static_cast<const char*>(tb.grad[(size_t)k * tb.n_seg + seg]) + ch.off * gsz;
+                    if (ch.seg & kSegVecFlag) sumsq_chunk_bf16_fast(f, q[0], g, ch.len);
+                    else                      sumsq_chunk<PREC>(q, g, ch.len, false);
+                }
+                q[1] = dd_add(DD{f.dn[0], 0.0}, DD{f.dn[1], 0.0});     // the chains hold exact sums
+                q[2] = dd_add(DD{f.dn[2], 0.0}, DD{f.dn[3], 0.0});
+            }
+        }
+        for (uint32_t c = c_begin; c < c_end && !fast_done; ++c) {
         const Chunk ch = tb.chunks[c];
         const uint32_t seg = ch.seg & ~kSegVecFlag;
         const bool vec = (ch.seg & kSegVecFlag) != 0;

@@ -35,7 +35,7 @@ __host__ __device__ __forceinline__ U32x4 philox4x32_10(U32x4 ctr, uint32_t k0, 
     return ctr;
 }
 
-// Algorithm 1: "b ~ U[0,1]; if b <= p".  One draw per (worker k, step t):
+// Algorithm 1's branch draw (a uniform variate compared with p).  One draw per (worker k, step t):
 // word 0 of Philox with counter (t_lo, t_hi, k, 0) and key (seed_lo, seed_hi),
 // compared with thr = floor(p * 2^32).
 __host__ __device__ __forceinline__ bool draw_pull(uint64_t seed, uint64_t t, uint32_t k, uint64_t thr)

@@ -43,6 +43,16 @@ def shard_ranges(numel: Sequence[int], rank: int, world: int, align: int = 1024)
     return pieces
 
 
+def shard_span(numel: Sequence[int], rank: int, world: int, align: int = 1024) -> Tuple[int, int]:
+    """[lo, hi) of the concatenated element index that `rank` owns (the range `shard_ranges` cuts up)."""
+    if world < 1 or not 0 <= rank < world or align < 1:
+        raise ValueError("need 0 <= rank < world and align >= 1")
+    total = int(sum(numel))
+    per = -(-total // world)
+    per = -(-per // align) * align
+    return min(total, rank * per), min(total, (rank + 1) * per)
+
+
 def shard_numel(numel: Sequence[int], rank: int, world: int, align: int = 1024) -> List[int]:
     """Element counts of the pieces of `shard_ranges` (the tensor list a rank's context is built on)."""
     return [b - a for _, a, b in shard_ranges(numel, rank, world, align)]

@@ -9,12 +9,14 @@ the outer-sync kernel once.  Achieved GB/s = algorithmic bytes / CUDA-event time
 where the inner bytes follow the decisions actually drawn in the timed steps
 (28 B per worker-element on a gradient step, 12 B on a pull; AdamW, fp32) and the
 outer bytes are (8K + 16) per parameter.  The average cost per step of a whole
-H-step cycle, (H * inner + outer) / H, is derived for every H.  Points that do not
-fit in 80 % of the free device memory are skipped.  Output: a Markdown table.
+H-step cycle, (H * inner + outer) / H, is derived for every H.  A point is run when its
+state plus a 4 GB margin fits in the device memory that is free once the previous point's
+buffers have been released; otherwise the row says what was free.  Output: a Markdown table.
 """
 from __future__ import annotations
 
 import argparse
+import gc
 import json
 import os
 import sys
@@ -61,9 +63,11 @@ def main() -> None:
         for logP in args.logP:
             Pn = 1 << logP
             need = K * Pn * 16 + 8 * Pn
+            gc.collect()
+            torch.cuda.empty_cache()
             free, _ = torch.cuda.mem_get_info(dev)
-            if need > 0.8 * free:
-                print(f"| {K} | 2^{logP} | {need / 1e9:.1f} | skipped: needs more than 80 % of the {free / 1e9:.0f} GB free |")
+            if need + (4 << 30) > free:
+                print(f"| {K} | 2^{logP} | {need / 1e9:.1f} | skipped: state + 4 GB margin exceeds the {free / 1e9:.0f} GB free |")
                 continue
             arena = ReplicaArena([Pn], K, precision=P.PREC_FP32, inner=P.INNER_ADAMW, device=dev)
             arena.model.normal_(0, 0.02)
@@ -102,8 +106,8 @@ def main() -> None:
                 row += [f"{(h * ms + outer[0]) / h:.4f}" for h in args.H]
                 print("| " + " | ".join(map(str, row)) + " |", flush=True)
                 ctx.destroy()
+                del ctx                                  # the context keeps its tensors alive
             del arena
-            torch.cuda.empty_cache()
 
 
 if __name__ == "__main__":

@@ -104,6 +104,47 @@ def test_sum_of_squares_is_exact_over_a_wide_dynamic_range():
     compare_state(gpu.state(), orc, exact=True)
 
 
+def _bf16_bits(a):
+    return W.bf16_bits_from_f32_host(np.asarray(a, dtype=np.float32))
+
+
+@pytest.mark.parametrize("kind", ["gaussian", "mostly_zero", "two_scales", "wide", "tiny_and_denormal", "one_outlier_late",
+                                  "infinite"])
+def test_bf16_sum_of_squares_is_exact_on_every_route(kind):
+    # bf16 gradients take plain binary64 chains whose exactness is tested after the run (ordinary data), send
+    # far-off elements through the double-double accumulator one by one, and redo an item in double-double when
+    # the test fails (data spread over many binades): all three routes must give the exactly rounded sum
+    numel = [8192 * 9 + 24, 40, 8192]
+    P = sum(numel)
+    cfg = _cfg(K=3, p=0.0, H=10**6, precision=1)
+    rng = np.random.default_rng(17)
+    gpu, orc = GpuRun(cfg, _x0(3, P), numel=numel), make_oracle(cfg, _x0(3, P))
+    gpu.set_grad_clip(1.0); orc.set_grad_clip(1.0)
+    for t in range(2):
+        z = rng.standard_normal((3, P))
+        if kind == "gaussian":
+            g = z * 0.01
+        elif kind == "mostly_zero":
+            g = np.where(rng.random((3, P)) < 0.97, 0.0, z * 0.01)
+        elif kind == "two_scales":                       # a few elements 2^-20 below the rest
+            g = np.where(rng.random((3, P)) < 0.001, z * 0.01 * 2.0 ** -20, z * 0.01)
+        elif kind == "wide":
+            g = z * np.exp2(rng.integers(-60, 60, (3, P)))
+        elif kind == "tiny_and_denormal":                # bf16 denormals (below 2^-126) among tiny normal values
+            g = z * np.exp2(rng.integers(-133, -120, (3, P)))
+        elif kind == "one_outlier_late":                 # the largest element arrives after the range was fixed
+            g = z * 0.01
+            g[:, P - 5] = 3.0e4
+        else:
+            g = z * 0.01
+            g[1, 12345] = np.inf
+        bits = _bf16_bits(g)
+        gpu.set_grads(bits); gpu.inner_step(1e-3, 16.0); orc.inner_step(bits, 1e-3, 16.0)
+        _check_norms(gpu, orc, range(3))
+    if kind != "infinite":
+        compare_state(gpu.state(), orc, exact=True)
+
+
 def test_threshold_above_every_norm_is_bitwise_the_unclipped_run_and_costs_one_more_launch():
     numel = RAGGED
     P = sum(numel)

@@ -1,12 +1,13 @@
-"""Full-coverage parity at benchmark size: EVERY element of the GPT-Neo-125M-shaped
-workload (K = 8, 125 M parameters, bf16 working copy + fp32 master) over its full
-512-step schedule against the CPU oracle.
+"""Full-coverage parity at benchmark size: EVERY element of a model-shaped workload, in
+the benchmark's launch configuration, over its full schedule against the CPU oracle.
 
-Takes several minutes and 25 GB of host memory, so it only runs when
-PALSGD_FULL_COVERAGE=1 is set; the default suite covers the same workload on a
-sample of indices (tests/test_gpu_configs.py).  Gradients are drawn on the device
-by torch's seeded generator (a harness input), copied to the host every step and
-fed to both sides.
+GPT-Neo-8M-shaped (K = 8, 256 steps, 4 outer syncs) and ResNet-50-shaped (K = 8, 128
+steps, 4 outer syncs) run in the default suite (well under a minute each).  The
+GPT-Neo-125M-shaped workload (bf16 working copy + fp32 master, 512 steps) takes several
+minutes and 25 GB of host memory, so it only runs when PALSGD_FULL_COVERAGE=1 is set;
+the default suite covers it on a sample of indices (tests/test_gpu_configs.py).
+Gradients are drawn on the device by torch's seeded generator (a harness input), copied
+to the host every step and fed to both sides.
 """
 import os
 import time
@@ -21,8 +22,10 @@ from _harness import GpuRun, make_oracle
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.skipif(os.environ.get("PALSGD_FULL_COVERAGE") != "1", reason="set PALSGD_FULL_COVERAGE=1 (slow)")
-@pytest.mark.parametrize("name", ["c3_gptneo125m_bf16"])
+_OPT_IN = pytest.mark.skipif(os.environ.get("PALSGD_FULL_COVERAGE") != "1", reason="set PALSGD_FULL_COVERAGE=1 (slow)")
+
+
+@pytest.mark.parametrize("name", ["c1_gptneo8m", "c2_resnet50", pytest.param("c3_gptneo125m_bf16", marks=_OPT_IN)])
 def test_every_element_full_schedule(name):
     import psutil
     cfg = W.get_config(name)

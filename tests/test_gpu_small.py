@@ -178,24 +178,25 @@ def test_run_to_run_determinism_and_launch_shape_independence():
             assert np.array_equal(outs[0][k], o[k]), k
 
 
-@pytest.mark.parametrize("variant,stages,cap", [(10, 0, 0), (11, 0, 0), (12, 0, 0), (10, 2, 3), (11, 3, 1), (12, 2, 2),
-                                                (3, 0, 0), (5, 0, 5), (7, 0, 0), (9, 0, 0), (13, 0, 0), (15, 0, 9), (18, 0, 0), (18, 0, 7)])
+@pytest.mark.parametrize("variant,cap", [(0, 0), (0, 5), (18, 0), (18, 7)])
 @pytest.mark.parametrize("inner,precision", [(0, 0), (1, 0), (0, 1), (1, 1)])
-def test_every_compiled_form_of_the_inner_kernel_matches_oracle(variant, stages, cap, inner, precision):
-    # 10/11: persistent shared-memory-ring form (full chunks through the ring, the rest by registers)
+def test_every_launch_form_of_the_inner_kernel_matches_oracle(variant, cap, inner, precision):
+    # 0: persistent grid that draws its work items from a queue; 18: one CTA per item; a capped grid
+    # strides over the items.  "misaligned": every buffer one element off 16-byte alignment, so each
+    # segment starts with a few elements on the scalar path and continues on the vector path
     numel = [4096 * 37 + 11, 5, 4096 * 2, 1001]
     P = sum(numel)
     cfg = _cfg(numel, K=5, H=3, T=7, p=0.3, inner=inner, precision=precision,
                momentum=0.9 if inner else 0.0)
     x0 = _x0(cfg.K, P, seed=5)
-    for layout in ("arena", "separate"):
+    for layout in ("arena", "separate", "misaligned"):
         gpu, orc = GpuRun(cfg, x0, numel=numel, layout=layout), make_oracle(cfg, x0)
-        gpu.lib.set_tuning(2, variant); gpu.lib.set_tuning(3, stages); gpu.lib.set_tuning(0, cap)
+        gpu.lib.set_tuning(2, variant); gpu.lib.set_tuning(0, cap)
         for t in range(cfg.T):
             g = _grads(cfg, P, t)
             gpu.set_grads(g); gpu.step(cfg.lr, cfg.eta); orc.step(g, cfg.lr, cfg.eta)
         compare_state(gpu.state(), orc, exact=True)
-        c = gpu.counters()                       # also raises if a bounded wait expired
+        c = gpu.counters()
         assert c["s"] == [int(v) for v in orc.s] and c["t"] == cfg.T
         assert gpu.guards_intact()
 
@@ -259,3 +260,44 @@ def test_step_host_transfers_no_gradient_for_workers_that_pull_and_splits_the_st
     compare_state(gpu.state(), orc, exact=True)
     assert gpu.lib.get_launch_count() - launches == 6 * cfg.K     # one launch per worker and step
     assert gpu.counters()["s"] == [int(v) for v in orc.s]
+
+
+def test_step_host_validates_the_result_pointers_before_anything_is_enqueued():
+    # a NULL entry in h_global on a step that ends with an outer sync: EINVAL, and nothing has moved
+    numel = [3000, 40]
+    P = sum(numel)
+    cfg = _cfg(numel, H=2)
+    x0 = _x0(cfg.K, P, same=True)
+    gpu = GpuRun(cfg, x0, numel=numel, layout="separate")
+    hg = torch.zeros((cfg.K, P), dtype=torch.float32).pin_memory()
+    hx = torch.empty(P, dtype=torch.float32).pin_memory()
+    starts = np.concatenate([[0], np.cumsum(numel)])
+    gp = gpu.lib.make_ptr_array([hg.data_ptr() + (k * P + int(starts[j])) * 4
+                                 for k in range(cfg.K) for j in range(len(numel))])
+    good = gpu.lib.make_ptr_array([hx.data_ptr() + int(starts[j]) * 4 for j in range(len(numel))])
+    bad = gpu.lib.make_ptr_array([hx.data_ptr(), 0])
+    assert gpu.lib.step_host(gp, cfg.lr, cfg.eta, bad, 0, gpu.stream) is False     # t = 1: no sync, pointers unused
+    before, launches = gpu.state(), gpu.lib.get_launch_count()
+    with pytest.raises(Exception) as e:
+        gpu.lib.step_host(gp, cfg.lr, cfg.eta, bad, 0, gpu.stream)                 # t = 2 would sync
+    assert getattr(e.value, "status", None) == -1
+    c = gpu.counters()                                                             # host and device agree: OK
+    assert c["t"] == 1 and c["n_outer"] == 0 and gpu.lib.get_launch_count() == launches
+    after = gpu.state()
+    for key in before:
+        assert np.array_equal(before[key], after[key]), key
+    assert gpu.lib.step_host(gp, cfg.lr, cfg.eta, good, 0, gpu.stream) is True     # the context is still usable
+    assert gpu.counters()["n_outer"] == 1
+
+
+def test_layout_report_counts_segments_and_chunks():
+    numel = [8192 * 2 + 5, 7, 0, 100]
+    cfg = _cfg(numel, inner=1, momentum=0.9)                     # 8192-element chunks
+    x0 = _x0(cfg.K, sum(numel))
+    # packed: the empty tensor (a NULL pointer) ends the first run of adjacent tensors
+    packed = GpuRun(cfg, x0, numel=numel, layout="arena").lib.get_layout()
+    assert packed == {"n_segments": 2, "n_chunks": 4, "chunk_elems": 8192}
+    shifted = GpuRun(cfg, x0, numel=numel, layout="misaligned").lib.get_layout()
+    assert shifted["n_segments"] == 2 and shifted["n_chunks"] == 6       # per segment a short scalar head, then aligned chunks
+    apart = GpuRun(cfg, x0, numel=numel, layout="separate").lib.get_layout()
+    assert apart["n_segments"] == 3 and apart["n_chunks"] == 5

@@ -1,0 +1,113 @@
+"""The outer synchronisation with the K workers spread over several contexts (one per GPU in a
+real deployment): palsgd_outer_partial -> sum of the exchange buffers -> palsgd_outer_finish.
+
+One GPU is at hand, so the several-rank case runs as several contexts on that GPU, one launch
+after the other (nothing waits on anything), with a plain tensor addition standing in for the
+all-reduce between two ranks (one commutative addition, so the result is the collective's).
+"""
+import numpy as np
+import pytest
+import torch
+
+import workloads as W
+from workloads.configs import WorkloadConfig
+from paper_2504_18454_b200.workers import DistributedPalsgd
+from _harness import GpuRun, compare_state, make_oracle
+
+pytestmark = pytest.mark.gpu
+
+RAGGED = [4096 * 3 + 5, 7, 1001, 0, 8192, 12]
+
+
+def _cfg(**kw):
+    base = dict(name="workers", shape=lambda: [], K=4, H=3, p=0.3, eta=16.0, lr=1e-3, T=7)
+    base.update(kw)
+    return WorkloadConfig(**base)
+
+
+def _grads(cfg, P, t, K_total):
+    g = np.stack([W.grads_host(P, cfg.grad_seed, t, k, cfg.grad_std) for k in range(K_total)])
+    return W.bf16_bits_from_f32_host(g) if cfg.precision == 1 else g
+
+
+@pytest.mark.parametrize("layout", ["arena", "separate", "misaligned"])
+@pytest.mark.parametrize("precision,outer_opt", [(0, 0), (1, 0), (0, 1), (1, 1)])
+def test_one_rank_is_bit_identical_to_the_plain_outer_sync(layout, precision, outer_opt):
+    cfg = _cfg(precision=precision, outer_opt=outer_opt, outer_lr=0.7 if outer_opt == 0 else 0.02)
+    P = sum(RAGGED)
+    rng = np.random.default_rng(3)
+    x0 = (rng.standard_normal((cfg.K, P)) * 0.02).astype(np.float32)
+    plain, orc = GpuRun(cfg, x0, numel=RAGGED, layout=layout), make_oracle(cfg, x0)
+    split = GpuRun(cfg, x0, numel=RAGGED, layout=layout)
+    exch = torch.zeros(split.lib.exchange_numel(), dtype=torch.float32, device=split.dev)
+    assert exch.numel() >= P
+    job = DistributedPalsgd(split.lib, exch, cfg.K, 0, 1, all_reduce_sum=lambda buf: None)
+    for t in range(cfg.T):
+        g = _grads(cfg, P, t, cfg.K)
+        plain.set_grads(g); split.set_grads(g)
+        plain.step(cfg.lr, cfg.eta); orc.step(g, cfg.lr, cfg.eta)
+        assert job.step(cfg.lr, cfg.eta, split.stream) == ((t + 1) % cfg.H == 0)
+    a, b = plain.state(), split.state()
+    for key in a:
+        assert np.array_equal(a[key], b[key]), key
+    compare_state(b, orc, exact=True)
+    assert split.counters()["n_outer"] == cfg.T // cfg.H and split.guards_intact()
+
+
+@pytest.mark.parametrize("inner,precision", [(0, 0), (1, 0), (0, 1)])
+def test_two_ranks_with_half_of_the_workers_each_match_one_oracle_with_all(inner, precision):
+    K_total, world = 6, 2
+    cfg = _cfg(K=K_total, inner=inner, precision=precision, momentum=0.9 if inner else 0.0, p=0.35)
+    P = sum(RAGGED)
+    x_init = (np.random.default_rng(9).standard_normal(P) * 0.02).astype(np.float32)
+    x0 = np.tile(x_init, (K_total, 1))
+    orc = make_oracle(cfg, x0)
+    local = cfg.with_(K=K_total // world)
+    ranks = [GpuRun(local, x0[: local.K], numel=RAGGED, layout="separate" if r else "arena") for r in range(world)]
+    for r, run in enumerate(ranks):
+        run.lib.set_worker_offset(r * local.K)
+    exch = [torch.zeros(run.lib.exchange_numel(), dtype=torch.float32, device=run.dev) for run in ranks]
+    for t in range(cfg.T):
+        g = _grads(cfg, P, t, K_total)
+        orc.step(g, cfg.lr, cfg.eta)
+        for r, run in enumerate(ranks):
+            run.set_grads(g[r * local.K:(r + 1) * local.K])
+            run.inner_step(cfg.lr, cfg.eta)
+            c = run.counters()                                  # the job's decisions, bit for bit
+            assert c["last_b"] == [int(v) for v in orc.last_b[r * local.K:(r + 1) * local.K]]
+        if (t + 1) % cfg.H == 0:
+            for run, e in zip(ranks, exch):
+                run.lib.outer_partial(e.data_ptr(), run.stream)
+            total = exch[0] + exch[1]                           # the all-reduce of two ranks: one addition
+            for run, e in zip(ranks, exch):
+                e.copy_(total)
+                run.lib.outer_finish(e.data_ptr(), K_total, run.stream)
+    states = [run.state() for run in ranks]
+    assert any(int(v) < cfg.T for v in orc.s) and orc.n_outer == 2
+    for key in ("xg", "u"):                                     # every rank holds the same global model
+        assert np.array_equal(states[0][key], states[1][key]), key
+    for r, (run, st) in enumerate(zip(ranks, states)):
+        sl = slice(r * local.K, (r + 1) * local.K)
+        assert run.counters()["s"] == [int(v) for v in orc.s[sl]]
+        # grouped by rank, the sum over k rounds differently from the oracle's ascending order:
+        # the parity bar (1e-6 relative, 1e-7 absolute floor) applies, not bitwise equality
+        class View:                                             # the oracle's rows of this rank
+            dtype = orc.dtype
+            x, m, v, xg, u, uv, xw = orc.x[sl], orc.m[sl], orc.v[sl], orc.xg, orc.u, None, None
+        compare_state({k: v for k, v in st.items() if k != "xw"}, View)
+        assert run.guards_intact()
+
+
+def test_argument_checks():
+    cfg = _cfg()
+    run = GpuRun(cfg, np.zeros((cfg.K, 100), dtype=np.float32), numel=[100])
+    buf = torch.zeros(run.lib.exchange_numel() + 4, dtype=torch.float32, device=run.dev)
+    for call in (lambda: run.lib.outer_partial(0, run.stream), lambda: run.lib.outer_finish(0, cfg.K, run.stream),
+                 lambda: run.lib.outer_finish(buf.data_ptr(), cfg.K - 1, run.stream)):
+        with pytest.raises(Exception) as e:
+            call()
+        assert getattr(e.value, "status", None) == -1
+    with pytest.raises(Exception) as e:
+        run.lib.outer_partial(buf.data_ptr() + 4, run.stream)
+    assert getattr(e.value, "status", None) == -2
+    assert run.counters()["n_outer"] == 0

@@ -1,7 +1,7 @@
 """Pins for the oracle's global-norm gradient clipping.
 
-The paper trains GPT-Neo with "gradient clipping enabled" (Appendix B) and says
-no more; the oracle takes the convention of the software the paper ran
+Appendix B states that the GPT-Neo runs clip their gradients and says no more
+(no threshold, no formula); the oracle takes the convention of the software the paper ran
 (PyTorch's clip_grad_norm_: coefficient max_norm / (norm + 1e-6), capped at 1,
 one norm over the worker's whole gradient).  Pinned here: the sum of squares
 against Python's exact summation, the clipped step against the library routine

@@ -20,7 +20,7 @@ import torch
 import paper_2504_18454_b200 as P
 import workloads as W
 from workloads.configs import WorkloadConfig
-from _harness import GpuRun
+from _harness import GpuRun, compare_state, make_oracle
 
 pytestmark = pytest.mark.gpu
 
@@ -85,6 +85,57 @@ def test_two_calls_in_a_row_match_the_ordinary_outer_sync(precision):
         st = tst.state()
         for k in range(K):
             assert np.array_equal(st["x"][k], st["xg"])        # every slot restarted from the global model
+
+
+@pytest.mark.parametrize("precision", [0, 1])
+def test_matches_the_cpu_oracle_directly(precision):
+    # the same comparison every other parity test makes: CUDA against the oracle, element by element,
+    # through two synchronisations with inner steps in between
+    numel = [8192 * 2 + 9, 33, 0, 4100]
+    Pn = int(sum(numel))
+    cfg = _cfg(K=4, precision=precision)
+    rng = np.random.default_rng(21)
+    x0 = (rng.standard_normal((cfg.K, Pn)) * 0.02).astype(np.float32)
+    run, orc = GpuRun(cfg, x0, numel=numel, layout="separate"), make_oracle(cfg, x0)
+    for rnd in range(2):
+        for t in range(cfg.T):
+            g = np.stack([W.grads_host(Pn, cfg.grad_seed, rnd * cfg.T + t, k, cfg.grad_std) for k in range(cfg.K)])
+            g = W.bf16_bits_from_f32_host(g) if precision == 1 else g
+            run.set_grads(g); run.inner_step(cfg.lr, cfg.eta); orc.inner_step(g, cfg.lr, cfg.eta)
+        _noalloc_sync(run, cfg)
+        orc.outer_sync()
+        compare_state(run.state(), orc, exact=True)
+    assert run.guards_intact()
+
+
+def test_refuses_a_capturing_stream():
+    # under capture the table copy and the kernel node would be replayed with whatever later calls
+    # left in the shared array, so the call must return ESTATE and enqueue nothing
+    dev = torch.device("cuda:0")
+    numel = [5000]
+    cfg = _cfg(K=2)
+    run = _diverged_run(cfg, numel, "arena", 3)
+    before = run.state()
+    side = torch.cuda.Stream(device=dev)
+    v = run.views
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        graph.capture_begin()
+        try:
+            with pytest.raises(P.PalsgdError) as e:
+                P.outer_sync_noalloc(K=cfg.K, numel=run.numel, params=v["param"], global_=v["global_"][0],
+                                     outer_mom=v["outer_mom"][0], stream=side.cuda_stream)
+        finally:
+            graph.capture_end()
+    assert e.value.status == -4
+    torch.cuda.synchronize(dev)
+    after = run.state()
+    for key in before:
+        assert np.array_equal(before[key], after[key]), key
+    _noalloc_sync(run, cfg)                                    # and the entry point still works afterwards
+    st = run.state()
+    for k in range(cfg.K):
+        assert np.array_equal(st["x"][k], st["xg"])
 
 
 def test_plain_averaging_and_non_nesterov_momentum():
