@@ -254,13 +254,17 @@ int launch_gradnorm(palsgd_ctx* ctx, bool ddp, cudaStream_t s)
     a.Kf = (float)ctx->cfg.K;
     a.k0 = ctx->k0;
     a.ddp = ddp ? 1u : 0u;
-    // chunks per work item: up to 8 (4 for the K-stream averaged form), fewer while that would leave
-    // under ~2048 items; fixed by the problem, so results never depend on the device or on tuning knobs
+    // chunks per group (the unit a CTA fetches at a time): up to 8 (4 for the K-stream averaged form), fewer
+    // while that would leave under ~2048 groups
     const uint32_t kitems = ddp ? 1u : ctx->cfg.K;
     const uint64_t items1 = (uint64_t)ctx->tb.n_chunks * kitems;
     a.group = (uint32_t)std::min<uint64_t>(ddp ? 4 : 8, std::max<uint64_t>(1, items1 / 2048));
     const uint64_t n_groups = (ctx->tb.n_chunks + a.group - 1) / a.group;
-    const unsigned grid = grid_for(n_groups * kitems, ctx->grid_cap_inner);
+    // a persistent grid: every CTA works for one worker and leaves one partial (3 CTAs per SM are resident)
+    int cap = ctx->sm_count > 0 ? ctx->sm_count * 3 : 444;
+    if (ctx->grid_cap_inner > 0) cap = std::min(cap, ctx->grid_cap_inner);
+    // (at least one CTA per worker, whatever the cap: a CTA serves a single worker)
+    const unsigned grid = std::max<unsigned>(grid_for(n_groups * kitems, cap), kitems);
     const bool bf = ctx->cfg.precision == PALSGD_PREC_BF16_MASTER;
     return launch_checked(ctx, [&] {
         if (bf) palsgd_gradnorm_kernel<1><<<grid, kThreads, 0, s>>>(a);

@@ -141,13 +141,13 @@ __device__ __forceinline__ void sumsq_chunk(DD (&q)[4], const void* g, uint32_t 
 // the start of the chunk and this thread's elements of the chunk are added in double-double.
 // Zeros, denormals and infinities need no special case (inf = inf keeps the chains equal).
 struct FastSq {
-    double dn[4], up[4];        // four independent chains (element position mod 4), rounded down / up
-    double ok[4];               // their (common) values at the start of the current chunk
+    double dn[2], up[2];        // two independent chains (even / odd element position), rounded down / up
+    double ok[2];               // their (common) values at the start of the current piece
 
     __device__ __forceinline__ void init()
     {
 #pragma unroll
-        for (int j = 0; j < 4; ++j) { dn[j] = 0.0; up[j] = 0.0; ok[j] = 0.0; }
+        for (int j = 0; j < 2; ++j) { dn[j] = 0.0; up[j] = 0.0; ok[j] = 0.0; }
     }
     __device__ __forceinline__ void add(int j, float g)
     {
@@ -159,9 +159,9 @@ struct FastSq {
     // false: the chains have been put back to where they were at that call
     __device__ __forceinline__ bool settle()
     {
-        const bool exact = dn[0] == up[0] && dn[1] == up[1] && dn[2] == up[2] && dn[3] == up[3];
+        const bool exact = dn[0] == up[0] && dn[1] == up[1];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
+        for (int j = 0; j < 2; ++j) {
             if (exact) ok[j] = dn[j];
             else { dn[j] = ok[j]; up[j] = ok[j]; }
         }
@@ -169,88 +169,130 @@ struct FastSq {
     }
 };
 
-// One 16-byte-aligned chunk of one bf16 gradient: this thread's groups of 8 into the fast chains, or,
-// if the chains' test fails for this chunk, once more into the double-double accumulator `slow`.
-__device__ __forceinline__ void sumsq_chunk_bf16_fast(FastSq& f, DD& slow, const void* g, uint32_t len)
+// One piece of a work item of the norm pass: `len` bf16 gradients at g.
+struct NormPiece { const void* g; uint32_t len; uint32_t vec; };
+constexpr uint32_t kNormGroupMax = 8;      // chunks per work item at most
+constexpr int kNormU = 4;                  // 128-bit loads per thread and piece
+
+// First kThreads * kNormU groups of 8 of a 16-byte-aligned piece into registers (zeros elsewhere).
+__device__ __forceinline__ void norm_piece_load(uint4 (&R)[kNormU], const NormPiece& p)
 {
-    constexpr int U = 4;
-    const uint4* g8 = static_cast<const uint4*>(g);
-    const uint32_t n8 = len >> 3;
-    for (uint32_t base = 0; base < n8; base += kThreads * U) {
-        uint4 R[U];
+    const uint4* g8 = static_cast<const uint4*>(p.g);
+    const uint32_t n8 = p.vec ? min(p.len >> 3, kThreads * (uint32_t)kNormU) : 0u;
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const uint32_t i = base + u * kThreads + threadIdx.x;
-            R[u] = i < n8 ? ld_stream(g8 + i) : make_uint4(0u, 0u, 0u, 0u);      // zeros add nothing
-        }
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            float v[8]; unpack8(R[u], v);
-#pragma unroll
-            for (int c = 0; c < 8; ++c) f.add(c & 3, v[c]);
-        }
+    for (int u = 0; u < kNormU; ++u) {
+        const uint32_t i = u * kThreads + threadIdx.x;
+        R[u] = i < n8 ? ld_stream(g8 + i) : make_uint4(0u, 0u, 0u, 0u);            // zeros add nothing
     }
-    if (!f.settle()) {                                      // rare; the data is still in cache
-        for (uint32_t i = threadIdx.x; i < n8; i += kThreads) {
-            float v[8]; unpack8(__ldg(g8 + i), v);
-#pragma unroll
-            for (int c = 0; c < 8; ++c) dd_square_in(slow, v[c]);
-        }
-    }
-    for (uint32_t i = (n8 << 3) + threadIdx.x; i < len; i += kThreads)
-        dd_square_in(slow, __bfloat162float(static_cast<const __nv_bfloat16*>(g)[i]));
 }
 
-// One launch ahead of a step whose gradients are clipped.  Work items: (chunk, worker) with the
-// worker index fastest (ddp = 0), or chunks (ddp = 1: the norm of the averaged gradient, formed
-// exactly as the DDP step forms it).  Every item leaves a double-double partial in
-// tb.norm_part (indexed [group * workers + worker]); the last CTA to finish adds the partials of each worker in item order and
-// writes sumsq and the clip coefficient to the device state.
+// The loaded groups into the fast chains; if the chains' test then fails, the chains are put back and
+// the same elements are added once more in double-double (rare; the data is still in cache).  Whatever
+// the registers did not cover (an unaligned piece, a piece longer than the registers, an odd tail)
+// goes through the double-double accumulator as well.
+__device__ __forceinline__ void norm_piece_consume(FastSq& f, DD& slow, const uint4 (&R)[kNormU], const NormPiece& p)
+{
+    const uint4* g8 = static_cast<const uint4*>(p.g);
+    const uint32_t n8_all = p.vec ? p.len >> 3 : 0u;
+    const uint32_t n8 = min(n8_all, kThreads * (uint32_t)kNormU);
+#pragma unroll
+    for (int u = 0; u < kNormU; ++u) {
+        float v[8]; unpack8(R[u], v);
+#pragma unroll
+        for (int c = 0; c < 8; ++c) f.add(c & 1, v[c]);
+    }
+    uint32_t redo_from = n8;                                // groups [redo_from, n8_all) go the slow way
+    if (!f.settle()) redo_from = 0;
+    for (uint32_t i = redo_from + threadIdx.x; i < n8_all; i += kThreads) {
+        float v[8]; unpack8(__ldg(g8 + i), v);
+#pragma unroll
+        for (int c = 0; c < 8; ++c) dd_square_in(slow, v[c]);
+    }
+    for (uint32_t i = (n8_all << 3) + threadIdx.x; i < p.len; i += kThreads)
+        dd_square_in(slow, __bfloat162float(static_cast<const __nv_bfloat16*>(p.g)[i]));
+}
+
+// All pieces of a work item, software-pipelined: the loads of piece c+1 are in flight while piece c
+// is being added up (the pieces' addresses were resolved beforehand, so nothing but the data itself
+// is waited for).
+__device__ __forceinline__ void norm_group_bf16_fast(FastSq& f, DD& slow, const NormPiece* pieces, uint32_t n)
+{
+    uint4 A[kNormU], B[kNormU];
+    norm_piece_load(A, pieces[0]);
+    for (uint32_t c = 0; c < n; c += 2) {
+        if (c + 1 < n) norm_piece_load(B, pieces[c + 1]);
+        norm_piece_consume(f, slow, A, pieces[c]);
+        if (c + 2 < n) norm_piece_load(A, pieces[c + 2]);
+        if (c + 1 < n) norm_piece_consume(f, slow, B, pieces[c + 1]);
+    }
+}
+
+// One launch ahead of a step whose gradients are clipped.  The grid is persistent (a few CTAs per
+// SM).  Every CTA works for ONE worker that takes a gradient step (ddp = 0), or for the one
+// averaged gradient (ddp = 1: formed exactly as the DDP step forms it): with n_act such workers,
+// CTA b serves the (b mod n_act)-th of them and walks over the groups of a.group consecutive
+// chunks  b / n_act, b / n_act + C, ...  (C = gridDim / n_act CTAs per worker), adding up in
+// registers across all of them, so that the CTA-wide reduction is paid once per CTA.  Every CTA
+// leaves one double-double partial in tb.norm_part[b]; the last CTA to finish adds the partials
+// of each worker (one warp per worker) and writes sumsq and the clip coefficient to the device
+// state.  The sums are exact up to the final rounding, so the result does not depend on how the
+// work was cut.
 template <int PREC>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 3)
 palsgd_gradnorm_kernel(const __grid_constant__ NormArgs a)
 {
-    __shared__ unsigned char s_pull[kMaxWorkers];
+    __shared__ unsigned char s_act[kMaxWorkers];            // the workers that take a gradient step, ascending
+    __shared__ unsigned int s_n_act;
     __shared__ DD s_warp[kThreads / 32];
     __shared__ const void* s_g[kMaxWorkers];
+    __shared__ NormPiece s_piece[kNormGroupMax];
     __shared__ unsigned int s_last;
     const Tables& tb = a.tb;
     const uint32_t K = tb.K;
     DevState* st = tb.st;
     const unsigned long long t = st->t;
-    const uint32_t Kitems = a.ddp ? 1u : K;
 
-    if (threadIdx.x < K) s_pull[threadIdx.x] = a.ddp ? 0 : draw_pull(a.seed, t, a.k0 + threadIdx.x, a.thr);
+    if (threadIdx.x == 0) {
+        unsigned int n = 0;
+        if (a.ddp) { s_act[0] = 0; n = 1; }
+        else for (uint32_t k = 0; k < K; ++k) if (!draw_pull(a.seed, t, a.k0 + k, a.thr)) s_act[n++] = (unsigned char)k;
+        s_n_act = n;
+    }
     __syncthreads();
+    const uint32_t n_act = s_n_act;
+    const uint32_t per_worker = n_act ? gridDim.x / n_act : 0u;        // CTAs per worker (the rest idle)
+    const uint32_t mine = n_act ? blockIdx.x % n_act : 0u;
+    const uint32_t lane_of_worker = n_act ? blockIdx.x / n_act : 0u;
+    const bool working = n_act && lane_of_worker < per_worker;
+    const uint32_t k = working ? s_act[mine] : 0u;
 
-    // Work item = a.group consecutive chunks of one worker: the per-thread sums run over the whole
-    // group, so the CTA-wide reduction (as costly as ~20 elements per thread) is paid once per group.
     const uint32_t n_groups = (tb.n_chunks + a.group - 1) / a.group;
-    const uint64_t n_items = (uint64_t)n_groups * Kitems;
     const size_t gsz = PREC ? 2 : 4;
-    for (uint64_t item = blockIdx.x; item < n_items; item += gridDim.x) {
-        const uint32_t k = (uint32_t)(item % Kitems);
-        const uint32_t c_begin = (uint32_t)(item / Kitems) * a.group;
+    DD q[4] = {{0.0, 0.0}, {0.0, 0.0}, {0.0, 0.0}, {0.0, 0.0}};
+    FastSq f; f.init();
+    for (uint32_t grp = lane_of_worker; working && grp < n_groups; grp += per_worker) {
+        const uint32_t c_begin = grp * a.group;
         const uint32_t c_end = min(c_begin + a.group, tb.n_chunks);
-        DD q[4] = {{0.0, 0.0}, {0.0, 0.0}, {0.0, 0.0}, {0.0, 0.0}};
-        bool fast_done = false;
         if (PREC == 1 && !a.ddp) {
-            // bf16 gradients: plain binary64 chains whose exactness is tested chunk by chunk
-            fast_done = true;
-            if (!s_pull[k]) {
-                FastSq f; f.init();
-                for (uint32_t c = c_begin; c < c_end; ++c) {
-                    const Chunk ch = tb.chunks[c];
-                    const uint32_t seg = ch.seg & ~kSegVecFlag;
-                    const char* g = static_cast<const char*>(tb.grad[(size_t)k * tb.n_seg + seg]) + ch.off * gsz;
-                    if (ch.seg & kSegVecFlag) sumsq_chunk_bf16_fast(f, q[0], g, ch.len);
-                    else                      sumsq_chunk<PREC>(q, g, ch.len, false);
-                }
-                q[1] = dd_add(DD{f.dn[0], 0.0}, DD{f.dn[1], 0.0});     // the chains hold exact sums
-                q[2] = dd_add(DD{f.dn[2], 0.0}, DD{f.dn[3], 0.0});
+            // bf16 gradients: plain binary64 chains whose exactness is tested piece by piece.  The pieces'
+            // addresses (chunk table -> pointer table, two dependent reads) are resolved for the whole
+            // group at once, so that the data loads of successive pieces can overlap.
+            __syncthreads();                                // the previous group's readers of s_piece
+            if (threadIdx.x < c_end - c_begin) {
+                const Chunk ch = tb.chunks[c_begin + threadIdx.x];
+                const uint32_t seg = ch.seg & ~kSegVecFlag;
+                s_piece[threadIdx.x] = NormPiece{static_cast<const char*>(tb.grad[(size_t)k * tb.n_seg + seg]) + ch.off * gsz,
+                                                 ch.len, (ch.seg & kSegVecFlag) ? 1u : 0u};
             }
+            __syncthreads();
+            norm_group_bf16_fast(f, q[0], s_piece, c_end - c_begin);
+            // the chains hold exact sums: fold them into the double-double total and start them afresh, so
+            // that the running sums stay small (the smaller they are, the smaller the elements they take exactly)
+            q[1] = dd_add(q[1], dd_add(DD{f.dn[0], 0.0}, DD{f.dn[1], 0.0}));
+            f.init();
+            continue;
         }
-        for (uint32_t c = c_begin; c < c_end && !fast_done; ++c) {
+        for (uint32_t c = c_begin; c < c_end; ++c) {
         const Chunk ch = tb.chunks[c];
         const uint32_t seg = ch.seg & ~kSegVecFlag;
         const bool vec = (ch.seg & kSegVecFlag) != 0;
@@ -287,16 +329,16 @@ palsgd_gradnorm_kernel(const __grid_constant__ NormArgs a)
                 }
                 dd_square_in(q[0], __fdiv_rn(sum, a.Kf));
             }
-        } else if (!s_pull[k]) {                            // a pulling worker's gradient is not used
+        } else {
             const char* g = static_cast<const char*>(tb.grad[(size_t)k * tb.n_seg + seg]) + ch.off * gsz;
             sumsq_chunk<PREC>(q, g, ch.len, vec);
         }
         }
-        const DD tot = dd_block_sum(dd_add(dd_add(q[0], q[1]), dd_add(q[2], q[3])), s_warp);
-        if (threadIdx.x == 0) tb.norm_part[item] = make_double2(tot.hi, tot.lo);
     }
+    const DD mine_tot = dd_block_sum(dd_add(dd_add(q[0], q[1]), dd_add(q[2], q[3])), s_warp);
+    if (threadIdx.x == 0) tb.norm_part[blockIdx.x] = make_double2(mine_tot.hi, mine_tot.lo);
 
-    // ---- the last CTA to finish reduces the partials
+    // ---- the last CTA to finish adds the partials: warp w takes the workers w, w + 8, ...
     __syncthreads();
     if (threadIdx.x == 0) {
         __threadfence();
@@ -306,22 +348,29 @@ palsgd_gradnorm_kernel(const __grid_constant__ NormArgs a)
     }
     __syncthreads();
     if (!s_last) return;
-    for (uint32_t k = 0; k < Kitems; ++k) {
-        if (!a.ddp && s_pull[k]) continue;                  // uniform over the CTA
+    const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (uint32_t w = warp; w < n_act; w += kThreads / 32) {
         DD acc{0.0, 0.0};
-        for (uint32_t c = threadIdx.x; c < n_groups; c += kThreads) {
-            const double2 p = __ldcg(tb.norm_part + (size_t)c * Kitems + k);
+        for (uint32_t j = lane; j < per_worker; j += 32) {   // CTA j * n_act + w worked for this worker
+            const double2 p = __ldcg(tb.norm_part + (size_t)j * n_act + w);
             acc = dd_add(acc, DD{p.x, p.y});
         }
-        const DD tot = dd_block_sum(acc, s_warp);
-        if (threadIdx.x == 0) {
-            const double sumsq = isfinite(tot.hi) ? __dadd_rn(tot.hi, tot.lo) : tot.hi;
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            DD o;
+            o.hi = __shfl_down_sync(0xFFFFFFFFu, acc.hi, off);
+            o.lo = __shfl_down_sync(0xFFFFFFFFu, acc.lo, off);
+            acc = dd_add(acc, o);
+        }
+        if (lane == 0) {
+            const double sumsq = isfinite(acc.hi) ? __dadd_rn(acc.hi, acc.lo) : acc.hi;
             const double coef = __ddiv_rn(a.max_norm, __dadd_rn(__dsqrt_rn(sumsq), 1e-6));
             const float clip = (float)(coef < 1.0 ? coef : 1.0);
             if (a.ddp) { for (uint32_t kk = 0; kk < K; ++kk) { st->sumsq[kk] = sumsq; st->clip[kk] = clip; } }
-            else       { st->sumsq[k] = sumsq; st->clip[k] = clip; }
+            else       { st->sumsq[s_act[w]] = sumsq; st->clip[s_act[w]] = clip; }
         }
     }
+    __syncthreads();
     if (threadIdx.x == 0) { st->done_norm = 0; __threadfence(); }
 }
 
