@@ -253,7 +253,6 @@ int launch_gradnorm(palsgd_ctx* ctx, bool ddp, cudaStream_t s)
     a.max_norm = ctx->max_grad_norm;
     a.Kf = (float)ctx->cfg.K;
     a.k0 = ctx->k0;
-    a.ddp = ddp ? 1u : 0u;
     // chunks per group (the unit a CTA fetches at a time): up to 8 (4 for the K-stream averaged form), fewer
     // while that would leave under ~2048 groups
     const uint32_t kitems = ddp ? 1u : ctx->cfg.K;
@@ -267,8 +266,10 @@ int launch_gradnorm(palsgd_ctx* ctx, bool ddp, cudaStream_t s)
     const unsigned grid = std::max<unsigned>(grid_for(n_groups * kitems, cap), kitems);
     const bool bf = ctx->cfg.precision == PALSGD_PREC_BF16_MASTER;
     return launch_checked(ctx, [&] {
-        if (bf) palsgd_gradnorm_kernel<1><<<grid, kThreads, 0, s>>>(a);
-        else    palsgd_gradnorm_kernel<0><<<grid, kThreads, 0, s>>>(a);
+        if (bf) { if (ddp) palsgd_gradnorm_kernel<1, 1><<<grid, kThreads, 0, s>>>(a);
+                  else     palsgd_gradnorm_kernel<1, 0><<<grid, kThreads, 0, s>>>(a); }
+        else    { if (ddp) palsgd_gradnorm_kernel<0, 1><<<grid, kThreads, 0, s>>>(a);
+                  else     palsgd_gradnorm_kernel<0, 0><<<grid, kThreads, 0, s>>>(a); }
     });
 }
 

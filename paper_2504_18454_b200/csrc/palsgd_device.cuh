@@ -126,7 +126,6 @@ struct NormArgs {
     double   max_norm;     // clip threshold
     float    Kf;
     uint32_t k0;           // the decision stream's index of local worker 0
-    uint32_t ddp;          // 0: per-worker norms (Algorithm 1 phase); 1: norm of the averaged gradient
     uint32_t group;        // consecutive chunks per work item (a function of the problem size only)
 };
 
