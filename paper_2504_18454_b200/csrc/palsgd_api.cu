@@ -354,9 +354,10 @@ extern "C" int palsgd_init(palsgd_ctx** out, const palsgd_config* cfg, size_t n_
     ctx->P = P;
     ctx->thr = threshold_of(cfg->p);
     ctx->outer_lr = cfg->outer_lr;
-    // work item of the outer kernel, measured on B200: with K + 2 streams per element few slots need
-    // larger slices to amortise the per-item prologue (K = 4: 0.88 -> 0.95 of the copy rate)
-    ctx->outer_sub_elems = K < 8 ? 4096u : kOuterSubElems;
+    // work item of the outer kernel, measured on B200: 1024 elements; for K = 5..7 (K + 2 streams per element,
+    // 4 CTAs per SM) larger items amortise the per-item prologue; K <= 4 runs the narrow-batch form of the
+    // kernel with 5 CTAs per SM, which does best with the small item (2048 for K <= 2)
+    ctx->outer_sub_elems = (K > 4 && K < 8) ? 4096u : K <= 2 ? 2048u : kOuterSubElems;
     ctx->ddp_sub_elems = bf ? 4096u : kDdpSubElems;
     ctx->h_grad_dev.assign(bufs->grad, bufs->grad + (size_t)K * n_tensors);
     ctx->h_global_dev.assign(bufs->global, bufs->global + n_tensors);
@@ -660,8 +661,9 @@ extern "C" int palsgd_outer_sync(palsgd_ctx* ctx, void* stream)
         const bool bcast = ctx->outer_variant != 1 && (int)stage_bytes <= ctx->smem_optin - 4096;   // measured best
         using OuterKernel = void (*)(const OuterArgs);
         OuterKernel kernel;
-        if (bcast) kernel = bf ? (oadam ? palsgd_outer_kernel<1, 1, 1> : palsgd_outer_kernel<1, 0, 1>)
-                               : (oadam ? palsgd_outer_kernel<0, 1, 1> : palsgd_outer_kernel<0, 0, 1>);
+        const bool few = ctx->cfg.K <= 4;                      // narrower load batches, one more CTA per SM
+        if (bcast) kernel = bf ? (oadam ? palsgd_outer_kernel<1, 1, 1> : few ? palsgd_outer_kernel<1, 0, 1, 0, 4> : palsgd_outer_kernel<1, 0, 1>)
+                               : (oadam ? palsgd_outer_kernel<0, 1, 1> : few ? palsgd_outer_kernel<0, 0, 1, 0, 4> : palsgd_outer_kernel<0, 0, 1>);
         else       kernel = bf ? (oadam ? palsgd_outer_kernel<1, 1, 0> : palsgd_outer_kernel<1, 0, 0>)
                                : (oadam ? palsgd_outer_kernel<0, 1, 0> : palsgd_outer_kernel<0, 0, 0>);
         if (bcast) { const int rc = ensure_dyn_smem(ctx, reinterpret_cast<const void*>(kernel), stage_bytes); if (rc) return rc; }
