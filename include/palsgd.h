@@ -331,7 +331,7 @@ int palsgd_get_layout(palsgd_ctx* ctx, uint64_t* n_segments, uint64_t* n_chunks,
  * INNER_VARIANT: 0 = the fused inner kernel as a persistent grid that draws its work items from a
  * queue in device memory (default); 18 = the same kernel with one CTA per work item.
  * OUTER_SUB_ELEMS: elements per work item of the outer kernel, a multiple of 1024; default 1024
- * (4096 for K = 5..7, 2048 for K <= 2).  DDP_SUB_ELEMS: the same for the DDP warm-up kernel.  Setting either rebuilds
+ * (4096 for K = 5..7, 2048 for K <= 2).  DDP_SUB_ELEMS: the same for the DDP warm-up kernel (default 1024).  Setting either rebuilds
  * a device table: the call synchronises the device and must not be made during stream capture.
  * DDP_VARIANT: how the DDP warm-up kernel writes its result to the K slots: 1 = 128-bit stores
  * by every thread, 2 = staged in shared memory and fanned out by bulk asynchronous stores;

@@ -358,7 +358,7 @@ extern "C" int palsgd_init(palsgd_ctx** out, const palsgd_config* cfg, size_t n_
     // 4 CTAs per SM) larger items amortise the per-item prologue; K <= 4 runs the narrow-batch form of the
     // kernel with 5 CTAs per SM, which does best with the small item (2048 for K <= 2)
     ctx->outer_sub_elems = (K > 4 && K < 8) ? 4096u : K <= 2 ? 2048u : kOuterSubElems;
-    ctx->ddp_sub_elems = bf ? 4096u : kDdpSubElems;
+    ctx->ddp_sub_elems = kDdpSubElems;
     ctx->h_grad_dev.assign(bufs->grad, bufs->grad + (size_t)K * n_tensors);
     ctx->h_global_dev.assign(bufs->global, bufs->global + n_tensors);
 

@@ -12,7 +12,7 @@ constexpr uint32_t kChunkElems  = 8192;    // default elements per chunk-table e
                                            // inner kernel (large: amortises the per-CTA prologue and tick)
 constexpr uint32_t kOuterSubElems = 1024;  // default work item of the outer kernel for K >= 8 (small: K+2
                                            // streams per element need many CTAs in flight)
-constexpr uint32_t kDdpSubElems = 1024;    // default work item of the DDP warm-up kernel in fp32 mode
+constexpr uint32_t kDdpSubElems = 1024;    // default work item of the DDP warm-up kernel (two stage buffers fit)
 constexpr uint32_t kSegVecFlag  = 0x80000000u;   // Chunk::seg bit: 16-byte vector path allowed
 
 // One work unit of the multi-tensor launch: `len` consecutive elements of

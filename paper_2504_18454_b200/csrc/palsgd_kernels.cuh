@@ -833,20 +833,23 @@ palsgd_ddp_kernel(const __grid_constant__ DdpArgs a)
                 if (INNER == 0) V = __ldcs(reinterpret_cast<const float4*>(s_v[0]) + i);
                 float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
                 for (uint32_t k0 = 0; k0 < K; k0 += B) {
-                    float4 R[B];
+                    // bf16 gradients stay packed in registers until they are added (half the registers)
+                    float4 R[PREC ? 1 : B]; uint2 H[PREC ? B : 1];
 #pragma unroll
                     for (int j = 0; j < B; ++j)
                         if (k0 + j < K) {
-                            if (PREC) { const uint2 h = __ldcs(static_cast<const uint2*>(s_g[k0 + j]) + i);
-                                        float f[4]; unpack4(h, f); R[j] = make_float4(f[0], f[1], f[2], f[3]); }
-                            else      { R[j] = __ldcs(static_cast<const float4*>(s_g[k0 + j]) + i); }
+                            if (PREC) H[j] = __ldcs(static_cast<const uint2*>(s_g[k0 + j]) + i);
+                            else      R[j] = __ldcs(static_cast<const float4*>(s_g[k0 + j]) + i);
                         }
 #pragma unroll
                     for (int j = 0; j < B; ++j)
                         if (k0 + j < K) {
-                            if (k0 + j == 0) acc = R[j];
-                            else { acc.x = __fadd_rn(acc.x, R[j].x); acc.y = __fadd_rn(acc.y, R[j].y);
-                                   acc.z = __fadd_rn(acc.z, R[j].z); acc.w = __fadd_rn(acc.w, R[j].w); }
+                            float4 r;
+                            if (PREC) { float f[4]; unpack4(H[j], f); r = make_float4(f[0], f[1], f[2], f[3]); }
+                            else      { r = R[j]; }
+                            if (k0 + j == 0) acc = r;
+                            else { acc.x = __fadd_rn(acc.x, r.x); acc.y = __fadd_rn(acc.y, r.y);
+                                   acc.z = __fadd_rn(acc.z, r.z); acc.w = __fadd_rn(acc.w, r.w); }
                         }
                 }
                 float4 G;
