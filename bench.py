@@ -484,6 +484,44 @@ def run_ours(args, cfg):
         ddp_ms = sum(evs[i].elapsed_time(evs[i + 1]) for i in range(8))
         ddp = {"ms": ddp_ms, "bytes": 8 * ddp_bytes_per_param(cfg) * Pn, "launches": 8}
 
+    # ---- the same two kernels on a ragged device layout (one allocation per worker and tensor), timed on their
+    # own after the main regions: frameworks hold their parameters that way, and the packed arenas above are
+    # the friendliest case for the multi-tensor metadata
+    ragged = None
+    if args.layout == "arena" and world == 1 and not args.no_ragged and len(numel) > 1:
+        arena2 = ReplicaArena(numel, K, precision=cfg.precision, inner=cfg.inner, device=dev, layout="separate")
+        for k in range(K):
+            arena2.write_flat(arena2.model_name, k, arena.read_flat(arena.model_name, k))
+            arena2.write_flat("grad", k, arena.read_flat("grad", k))
+        ctx2 = arena2.make_context(
+            stream=stream, H=1 << 40, p=cfg.p, beta1=cfg.beta1, beta2=cfg.beta2, eps=cfg.eps,
+            weight_decay=cfg.weight_decay, momentum=cfg.momentum, outer_lr=cfg.outer_lr,
+            outer_momentum=cfg.outer_momentum, outer_nesterov=cfg.outer_nesterov, seed=cfg.decision_seed)
+        n_in, n_out = 16, 4
+        for _ in range(3):
+            ctx2.inner_step(cfg.lr, cfg.eta, stream)
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(n_in + 1)]
+        ev[0].record()
+        for i in range(n_in):
+            ctx2.inner_step(cfg.lr, cfg.eta, stream); ev[i + 1].record()
+        oev = []
+        for i in range(n_out + 1):
+            for _ in range(2):
+                ctx2.inner_step(cfg.lr, cfg.eta, stream)
+            e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+            e0.record(); ctx2.outer_sync(stream); e1.record()
+            if i > 0:
+                oev.append((e0, e1))
+        torch.cuda.synchronize(dev)
+        in_ms = sum(ev[i].elapsed_time(ev[i + 1]) for i in range(n_in))
+        in_bytes = sum(inner_bytes_per_element(cfg, bool(P.decision(cfg.decision_seed, 3 + i, k, cfg.p)))
+                       for i in range(n_in) for k in range(K)) * Pn
+        out_ms = sum(a.elapsed_time(b) for a, b in oev)
+        ragged = {"layout": "separate", **ctx2.get_layout(), "inner_ms": in_ms, "inner_bytes": in_bytes, "n_inner": n_in,
+                  "outer_ms": out_ms, "outer_bytes": n_out * outer_bytes_per_param(cfg) * Pn, "n_outer": n_out}
+        ctx2.destroy()
+        del ctx2, arena2
+
     # ---- max over ranks
     ms_total, ms_e2e_max = max_over_ranks([ms_total, e2e["ms"] if e2e else 0.0], world, dev)
     if e2e:
@@ -516,6 +554,17 @@ def run_ours(args, cfg):
             "roofline_ddp": (roofline_entry("palsgd_ddp_kernel", "ddp", cfg, peak, peak_src, ddp["ms"], ddp["bytes"],
                                             ddp["launches"], units_per_launch=Pn,
                                             note="timed outside the step loop; not part of value") if ddp else None),
+            "ragged_layout": ({"layout": ragged["layout"], "n_segments": ragged["n_segments"],
+                               "n_chunks": ragged["n_chunks"],
+                               "roofline": roofline_entry("palsgd_inner_kernel", "inner", cfg, peak, peak_src,
+                                                          ragged["inner_ms"], ragged["inner_bytes"], ragged["n_inner"],
+                                                          traffic=None),
+                               "roofline_outer": roofline_entry("palsgd_outer_kernel", "outer", cfg, peak, peak_src,
+                                                                ragged["outer_ms"], ragged["outer_bytes"],
+                                                                ragged["n_outer"], units_per_launch=Pn, traffic=None),
+                               "note": "the same kernels over one allocation per (buffer kind, worker, tensor); "
+                                       "timed on their own after the main regions; not part of value"}
+                              if ragged else None),
             "graph_cycle": graph_cycle,
             "cpu_baseline": cpu_baseline,
             "e2e": ({"value": K * P_job * e2e["steps"] / (e2e["ms"] * 1e-3), "unit": UNIT,
@@ -550,6 +599,8 @@ def main():
     ap.add_argument("--outer-launches", type=int, default=8,
                     help="outer-sync launches timed on their own after the step loop")
     ap.add_argument("--no-outer", action="store_true", help="skip the separate timing of the outer-sync kernel")
+    ap.add_argument("--no-ragged", action="store_true",
+                    help="skip the separate timing of the inner and outer kernels on the one-allocation-per-tensor layout")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="skip the separate timing of the graph-captured cycle")

@@ -57,3 +57,15 @@ def test_bench_runs_on_the_ragged_layouts(layout):
     assert d["config"]["layout"] == layout
     assert d["config"]["n_segments"] == (99 if layout == "separate" else 1)
     assert d["roofline"]["achieved"] > 0 and d["roofline_outer"]["achieved"] > 0 and d["e2e"]["value"] > 0
+
+
+def test_default_layout_run_also_times_the_ragged_layout():
+    out = _run(["bench.py", "--workload", "c1_gptneo8m", "--steps", "4", "--warmup", "3", "--no-e2e",
+                "--no-cpu-baseline", "--no-graph", "--no-ddp"])
+    d = json.loads([l for l in out.splitlines() if l.startswith("{")][-1])
+    rg = d["ragged_layout"]
+    assert d["config"]["layout"] == "arena" and d["config"]["n_segments"] == 1
+    assert rg["layout"] == "separate" and rg["n_segments"] == 99
+    assert rg["roofline"]["launches"] == 16 and rg["roofline"]["achieved"] > 0 and rg["roofline"]["traffic"] is None
+    assert rg["roofline_outer"]["launches"] == 4 and rg["roofline_outer"]["achieved"] > 0
+    assert d["gpu_launches"] == 4                      # the extra region is not part of the timed step loop
