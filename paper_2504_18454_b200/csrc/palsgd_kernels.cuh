@@ -591,7 +591,6 @@ palsgd_outer_kernel(const __grid_constant__ OuterArgs a)
     const uint32_t K = tb.K;
     const uint32_t stage_bytes = a.sub_elems * (8u + (OOPT ? 4u : 0u) + (PREC ? 2u : 0u));
     const bool issuer = BCAST && threadIdx.x <= K;         // thread k < K: slot k's copies; thread K: x_g and u
-    const uint32_t Ksum = SUMIN ? 0u : K;                  // slots summed here (none when the sum comes in ready-made)
 
     ItemWalk walk{s_slots, a.dynamic, tb.st, 0, 0};
     for (uint32_t item = walk.first(); item < a.n_items; item = walk.next()) {
@@ -630,7 +629,7 @@ palsgd_outer_kernel(const __grid_constant__ OuterArgs a)
                         acc = make_float4(__ldcs(sum_src + 4 * i), __ldcs(sum_src + 4 * i + 1),
                                           __ldcs(sum_src + 4 * i + 2), __ldcs(sum_src + 4 * i + 3));
                 }
-                for (uint32_t k0 = 0; k0 < Ksum; k0 += B) {
+                for (uint32_t k0 = 0; !SUMIN && k0 < K; k0 += B) {
                     float4 R[B];
 #pragma unroll
                     for (int j = 0; j < B; ++j)
@@ -698,7 +697,7 @@ palsgd_outer_kernel(const __grid_constant__ OuterArgs a)
         }
         for (uint32_t i = done + threadIdx.x; i < ch.len; i += kThreads) {
             float sum = SUMIN ? sum_src[i] : s_x[0][i];
-            for (uint32_t k = 1; k < Ksum; ++k) sum = __fadd_rn(sum, s_x[k][i]);
+            for (uint32_t k = 1; !SUMIN && k < K; ++k) sum = __fadd_rn(sum, s_x[k][i]);
             float ui = um[i], xn;
             if (OOPT) { float vi = uv[i]; xn = outer_elem_adamw(sum, a.Kf, xg[i], ui, vi, os); uv[i] = vi; }
             else      { xn = outer_elem(sum, a.Kf, xg[i], ui, a.mu, a.lr, a.nesterov); }

@@ -132,6 +132,11 @@ def test_later_entry_points_reject_a_null_context():
     assert L.palsgd_cycle_launch(None, None) == -1
     assert L.palsgd_step_host(None, None, 1e-3, 1.0, None, None, None, None) == -1
     assert L.palsgd_set_tuning(None, 0, 0) == -1
+    assert L.palsgd_get_layout(None, None, None, None) == -1
+    assert L.palsgd_exchange_numel(None, None) == -1
+    assert L.palsgd_set_worker_offset(None, 0) == -1
+    assert L.palsgd_outer_partial(None, None, None) == -1
+    assert L.palsgd_outer_finish(None, None, 1, None) == -1
 
 
 @pytest.mark.parametrize("over", [dict(outer_opt=2), dict(outer_opt=1),                      # AdamW outer without outer_v
