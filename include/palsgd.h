@@ -325,7 +325,8 @@ int palsgd_get_launch_count(palsgd_ctx* ctx, uint64_t* n_launches);
  * per worker each) and the chunk size.  Any output pointer may be NULL.  Errors: EINVAL. */
 int palsgd_get_layout(palsgd_ctx* ctx, uint64_t* n_segments, uint64_t* n_chunks, uint32_t* chunk_elems);
 
-/* Launch-shape knobs (advanced; results never depend on them).
+/* Launch-shape knobs (advanced; results never depend on them).  Setting any of them drops a cycle recorded by
+ * palsgd_cycle_capture (palsgd_cycle_launch then returns ESTATE until the cycle is captured again).
  * *_GRID_CAP: the largest grid a launch may use, CTAs looping over work items
  * beyond it; 0 (default) = one CTA per work item.
  * INNER_VARIANT: 0 = the fused inner kernel as a persistent grid that draws its work items from a

@@ -12,6 +12,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <string>
 #include <vector>
@@ -75,8 +76,7 @@ struct palsgd_ctx {
     cudaGraphExec_t cycle_exec = nullptr;         // captured H-step cycle (palsgd_cycle_capture) or nullptr
     uint64_t cycle_launches = 0;                  // kernels inside one captured cycle
     int sm_count = 0, smem_optin = 0;             // device attributes read at init
-    // kernels whose dynamic-shared-memory limit has been raised on this context's device, with the limit set
-    std::vector<std::pair<const void*, int>> smem_attr;
+    int device = 0;                               // the device that was current at palsgd_init
     bool failed = false;                          // a CUDA call failed midway through an earlier entry point:
                                                   // device state and host mirrors may disagree, so every later
                                                   // call that would touch them returns PALSGD_ESTATE
@@ -226,20 +226,26 @@ OuterArgs outer_args(const palsgd_ctx* ctx)
     return a;
 }
 
-// Raise a kernel's dynamic-shared-memory limit once per context (the attribute belongs to the
-// function on the context's device; setting it again on every launch costs a few microseconds).
+// Raise a kernel's dynamic-shared-memory limit when a launch needs more than the limit in force.  The
+// attribute belongs to the function on a device, not to a context: the limits set so far are kept per
+// (device, kernel) for the whole process and only ever raised, so that contexts with different item sizes
+// cannot lower each other's limit, and the runtime call is made once instead of on every launch.
 int ensure_dyn_smem(palsgd_ctx* ctx, const void* kernel, size_t bytes)
 {
     if (bytes + 4096 <= 48 * 1024) return PALSGD_OK;         // static + dynamic within the default limit
-    for (auto& kv : ctx->smem_attr)
-        if (kv.first == kernel) {
-            if (kv.second >= (int)bytes) return PALSGD_OK;
+    struct Entry { int dev; const void* kernel; int bytes; };
+    static std::mutex mu;
+    static std::vector<Entry> limits;
+    std::lock_guard<std::mutex> lock(mu);
+    for (Entry& e : limits)
+        if (e.dev == ctx->device && e.kernel == kernel) {
+            if (e.bytes >= (int)bytes) return PALSGD_OK;
             PALSGD_CUDA(ctx, cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes));
-            kv.second = (int)bytes;
+            e.bytes = (int)bytes;
             return PALSGD_OK;
         }
     PALSGD_CUDA(ctx, cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes));
-    ctx->smem_attr.emplace_back(kernel, (int)bytes);
+    limits.push_back(Entry{ctx->device, kernel, (int)bytes});
     return PALSGD_OK;
 }
 
@@ -440,6 +446,7 @@ extern "C" int palsgd_init(palsgd_ctx** out, const palsgd_config* cfg, size_t n_
     {
         int dev = 0;
         if (cudaGetDevice(&dev) == cudaSuccess) {
+            ctx->device = dev;
             cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, dev);
             cudaDeviceGetAttribute(&ctx->smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
         }
@@ -1015,6 +1022,8 @@ extern "C" int palsgd_get_layout(palsgd_ctx* ctx, uint64_t* n_segments, uint64_t
 extern "C" int palsgd_set_tuning(palsgd_ctx* ctx, int knob, int64_t value)
 {
     if (!ctx || value < 0 || value > 0x7FFFFFFF) return PALSGD_EINVAL;
+    // a recorded cycle holds the launch shapes (and item-table addresses) of the moment it was captured
+    if (ctx->cycle_exec) { cudaGraphExecDestroy(ctx->cycle_exec); ctx->cycle_exec = nullptr; }
     switch (knob) {
         case PALSGD_TUNE_INNER_GRID_CAP: ctx->grid_cap_inner = (int)value; return PALSGD_OK;
         case PALSGD_TUNE_OUTER_GRID_CAP: ctx->grid_cap_outer = (int)value; return PALSGD_OK;

@@ -96,3 +96,25 @@ def test_cycle_state_errors():
     with pytest.raises(P.PalsgdError) as e:
         adam_outer.lib.cycle_capture(1e-3, 16.0)
     assert e.value.status == -6
+
+
+def test_changing_a_launch_knob_drops_the_recorded_cycle():
+    # the recording holds launch shapes and item-table addresses; a knob that rebuilds a table would leave
+    # it pointing at freed memory, so any knob change invalidates it
+    numel = [5000, 300]
+    cfg = _cfg(H=2)
+    x0 = _x0(cfg.K, 5300)
+    a, orc = GpuRun(cfg, x0, numel=numel), make_oracle(cfg, x0)
+    g = _grads(cfg, 5300, 0)
+    a.set_grads(g)
+    a.lib.cycle_capture(cfg.lr, cfg.eta)
+    a.lib.cycle_launch(a.stream)
+    a.lib.set_tuning(P.TUNE_OUTER_SUB_ELEMS, 2048)
+    with pytest.raises(P.PalsgdError) as e:
+        a.lib.cycle_launch(a.stream)
+    assert e.value.status == -4
+    a.lib.cycle_capture(cfg.lr, cfg.eta)              # recorded again with the new table
+    a.lib.cycle_launch(a.stream)
+    for _ in range(2 * cfg.H):
+        orc.step(g, cfg.lr, cfg.eta)
+    compare_state(a.state(), orc, exact=True)

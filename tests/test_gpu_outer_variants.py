@@ -146,3 +146,23 @@ def test_every_form_of_the_outer_kernel_matches_oracle(variant, sub, dyn, precis
             gpu.set_grads(g); gpu.step(cfg.lr, cfg.eta); orc.step(g, cfg.lr, cfg.eta)
         compare_state(gpu.state(), orc, exact=True)
         assert gpu.guards_intact()
+
+
+@pytest.mark.gpu
+def test_two_contexts_with_different_item_sizes_do_not_lower_each_others_shared_memory_limit():
+    # the dynamic-shared-memory limit belongs to the kernel on the device: the context with the larger
+    # stage sets it first, the one with the smaller stage must not lower it
+    numel = [16384 * 2 + 40]
+    Pn = sum(numel)
+    cfg = _cfg(K=3, H=1, T=3)
+    x0 = _x0(cfg.K, Pn, seed=4)
+    big, small, orc = GpuRun(cfg, x0, numel=numel), GpuRun(cfg, x0, numel=numel), make_oracle(cfg, x0)
+    big.lib.set_tuning(5, 16384)          # 128 KB of stage per CTA
+    small.lib.set_tuning(5, 8192)         # 64 KB
+    for t in range(cfg.T):
+        g = _grads(cfg, Pn, t)
+        orc.step(g, cfg.lr, cfg.eta)
+        big.set_grads(g); small.set_grads(g)
+        big.step(cfg.lr, cfg.eta); small.step(cfg.lr, cfg.eta)      # H = 1: big, small, big, small, ... outer syncs
+    compare_state(big.state(), orc, exact=True)
+    compare_state(small.state(), orc, exact=True)
