@@ -27,8 +27,14 @@
  *     Successive calls on one context must be stream-ordered with each other.
  *   - A context is not thread-safe; distinct contexts are independent.
  *   - Buffers need only natural element alignment.  Tensors whose every buffer
- *     is 16-byte aligned take the 128-bit vector path; others a scalar path
- *     with identical results.
+ *     is 16-byte aligned take the 128-bit vector path; so do tensors whose
+ *     buffers all become 16-byte aligned after the same small number of leading
+ *     elements (a packed list at an odd offset), behind a scalar head of those
+ *     elements; anything else takes a scalar path.  Results are identical.
+ *   - Arguments are checked before anything is enqueued: an EINVAL / EALIGN call
+ *     has changed nothing.  If a CUDA call fails in the middle of an entry point
+ *     (PALSGD_ECUDA), the context is marked failed and every later call that
+ *     would read or advance its state returns PALSGD_ESTATE; destroy it.
  *   - Arithmetic: every element operation is one IEEE binary32 operation in the
  *     order documented at each call (no fused multiply-add, round-to-nearest
  *     division and square root).  Scalars (step sizes, bias corrections) are
@@ -123,7 +129,8 @@ int palsgd_init(palsgd_ctx** out, const palsgd_config* cfg, size_t n_tensors,
  * One pass of Algorithm 1's inner loop body for all K workers, ONE kernel launch (one
  * more, ahead of it, while gradient clipping is on: see palsgd_set_grad_clip).
  * For worker k the kernel draws b_k^(t), Algorithm 1's uniform variate compared with p: the first word r of
- * Philox4x32-10 with key (seed_lo, seed_hi) and counter (t_lo, t_hi, k, 0);
+ * Philox4x32-10 with key (seed_lo, seed_hi) and counter (t_lo, t_hi, k0 + k, 0), k0 the worker
+ * offset (0 unless palsgd_set_worker_offset was called);
  * b = (r < floor(p * 2^32)).  One draw per (worker, step) for the whole model.
  *   b = 1, Eq. (2):  d = x - x_g;  x = x - beta * d,   beta = fl32(alpha_t*eta_t/p).
  *          Gradient, moments and s_k are not touched.
@@ -275,7 +282,8 @@ int palsgd_cycle_launch(palsgd_ctx* ctx, void* stream);
  * of the inner step that belongs to worker k is launched when its gradient has arrived
  * (K launches per step; with gradient clipping on, or K = 1, one launch after all copies).
  * Errors: as palsgd_step; EINVAL for a NULL gradient pointer of a non-empty tensor of a
- * worker that takes a gradient step.
+ * worker that takes a gradient step, and for a NULL entry of h_global (non-empty tensor) on a
+ * step that ends with the outer sync -- both found before anything is enqueued.
  */
 int palsgd_step_host(palsgd_ctx* ctx, const void* const* h_grad, double lr_t, double eta_t,
                      float* const* h_global, uint8_t* h_decisions, int* synced, void* stream);
