@@ -139,7 +139,7 @@ def _state_struct(real):
             ("sumsq", C.POINTER(C.c_double)), ("clipc", C.POINTER(C.c_double)),
             ("outer_opt", C.c_int32), ("outer_beta1", C.c_double), ("outer_beta2", C.c_double),
             ("outer_eps", C.c_double), ("outer_weight_decay", C.c_double), ("uv", ptr),
-            ("opow1", C.c_double), ("opow2", C.c_double),
+            ("opow1", C.c_double), ("opow2", C.c_double), ("sum_groups", C.c_uint32),
         ]
 
     return State
@@ -200,7 +200,7 @@ class Oracle:
             sumsq=p_(self.sumsq, C.c_double), clipc=p_(self.clipc, C.c_double),
             outer_opt=int(outer_opt), outer_beta1=outer_beta1, outer_beta2=outer_beta2,
             outer_eps=outer_eps, outer_weight_decay=outer_weight_decay,
-            uv=p_(self.uv, ct) if self.uv is not None else None, opow1=1.0, opow2=1.0)
+            uv=p_(self.uv, ct) if self.uv is not None else None, opow1=1.0, opow2=1.0, sum_groups=0)
         L = lib()
         sfx = dtype
         self._init = getattr(L, f"palsgd_oracle_init_{sfx}")
@@ -228,6 +228,16 @@ class Oracle:
     @property
     def n_outer(self) -> int:
         return int(self._st.n_outer)
+
+    # workers spread over several machines ----------------------------------
+    def set_sum_groups(self, groups: int) -> None:
+        """Form the outer sync's sum over the K workers in two levels: `groups` machines of K/groups
+        consecutive workers each add up their own workers first (ascending), then the partial sums are
+        added in ascending order of the machines.  0 or 1: one level, ascending k."""
+        groups = int(groups)
+        if groups > 1 and self.K % groups != 0:
+            raise ValueError("the workers do not divide evenly over the groups")
+        self._st.sum_groups = groups
 
     # schedules -----------------------------------------------------------
     def set_outer_lr(self, lr: float) -> None:

@@ -83,6 +83,11 @@ typedef struct {
     double    outer_beta1, outer_beta2, outer_eps, outer_weight_decay;
     REAL     *uv;            /* [P] second outer moment (outer_opt = 1) or NULL    */
     double    opow1, opow2;  /* outer_beta1^n_outer, outer_beta2^n_outer           */
+    /* Workers spread over G machines (the paper's own deployment: Algorithm 1's All-Reduce across
+     * workers; Sec. 2.2: an average).  The sum over the K workers is then formed in two levels: each
+     * machine adds up its own K/G consecutive workers in ascending order, and the G partial sums are
+     * added in ascending order of the machines.  0 or 1 = one level, ascending k (K workers on one GPU). */
+    uint32_t  sum_groups;
 } FN(state);
 
 static uint16_t to_bf16(REAL a)
@@ -276,7 +281,16 @@ void FN(outer_sync)(FN(state) *st)
     #pragma omp parallel for schedule(static)
     for (int64_t i = 0; i < (int64_t)P; ++i) {
         REAL sum = st->x[i];
-        for (uint32_t k = 1; k < K; ++k) sum = sum + st->x[(size_t)k * P + i];
+        if (st->sum_groups > 1) {                        /* per machine first, then across machines */
+            const uint32_t per = K / st->sum_groups;
+            for (uint32_t gi = 0; gi < st->sum_groups; ++gi) {
+                REAL part = st->x[(size_t)(gi * per) * P + i];
+                for (uint32_t k = gi * per + 1; k < (gi + 1) * per; ++k) part = part + st->x[(size_t)k * P + i];
+                sum = gi == 0 ? part : sum + part;
+            }
+        } else {
+            for (uint32_t k = 1; k < K; ++k) sum = sum + st->x[(size_t)k * P + i];
+        }
         REAL xbar  = sum / (REAL)K;
         REAL delta = st->xg[i] - xbar;
         if (st->outer_opt == 1) {
