@@ -163,7 +163,7 @@ class Oracle:
                  outer_nesterov: bool = True, seed: int = 0, precision: int = 0,
                  max_grad_norm: float = 0.0, outer_opt: int = 0, outer_beta1: float = 0.9,
                  outer_beta2: float = 0.999, outer_eps: float = 1e-8, outer_weight_decay: float = 0.0,
-                 dtype: str = "f32"):
+                 sum_groups: int = 0, dtype: str = "f32"):
         x0 = np.asarray(x0)
         assert x0.ndim == 2 and x0.shape[0] == K, x0.shape
         self.dtype = dtype
@@ -201,6 +201,8 @@ class Oracle:
             outer_opt=int(outer_opt), outer_beta1=outer_beta1, outer_beta2=outer_beta2,
             outer_eps=outer_eps, outer_weight_decay=outer_weight_decay,
             uv=p_(self.uv, ct) if self.uv is not None else None, opow1=1.0, opow2=1.0, sum_groups=0)
+        self.K = int(K)
+        self.set_sum_groups(sum_groups)          # before the initial global model is formed
         L = lib()
         sfx = dtype
         self._init = getattr(L, f"palsgd_oracle_init_{sfx}")
@@ -231,9 +233,10 @@ class Oracle:
 
     # workers spread over several machines ----------------------------------
     def set_sum_groups(self, groups: int) -> None:
-        """Form the outer sync's sum over the K workers in two levels: `groups` machines of K/groups
-        consecutive workers each add up their own workers first (ascending), then the partial sums are
-        added in ascending order of the machines.  0 or 1: one level, ascending k."""
+        """Form the sum over the K workers (initial global model, outer sync) in two levels: `groups`
+        machines of K/groups consecutive workers each add up their own workers first (ascending), then
+        the partial sums are added in ascending order of the machines.  0 or 1: one level, ascending k.
+        The constructor's `sum_groups` applies it to the initial global model as well."""
         groups = int(groups)
         if groups > 1 and self.K % groups != 0:
             raise ValueError("the workers do not divide evenly over the groups")

@@ -106,18 +106,36 @@ static void refresh_working(FN(state) *st, uint32_t k)
     for (int64_t i = 0; i < (int64_t)st->P; ++i) xw[i] = to_bf16(x[i]);
 }
 
+/* Sum of the K local models at element i: ascending k, or (sum_groups > 1) per machine first and
+ * then across the machines, both ascending. */
+static REAL sum_over_workers(const FN(state) *st, size_t i)
+{
+    const uint32_t K = st->K;
+    const size_t P = st->P;
+    REAL sum = st->x[i];
+    if (st->sum_groups > 1) {
+        const uint32_t per = K / st->sum_groups;
+        for (uint32_t gi = 0; gi < st->sum_groups; ++gi) {
+            REAL part = st->x[(size_t)(gi * per) * P + i];
+            for (uint32_t k = gi * per + 1; k < (gi + 1) * per; ++k) part = part + st->x[(size_t)k * P + i];
+            sum = gi == 0 ? part : sum + part;
+        }
+    } else {
+        for (uint32_t k = 1; k < K; ++k) sum = sum + st->x[(size_t)k * P + i];
+    }
+    return sum;
+}
+
 /* Set-up: x_g = (1/K) sum_k x_k (Sec. 2.2 average; Algorithm 1 starts every
- * worker from the same x^(0), for which this is x^(0) itself), all optimizer
- * state zero, counters zero. */
+ * worker from the same x^(0), for which this is x^(0) up to the rounding of the
+ * sum and the division), all optimizer state zero, counters zero. */
 void FN(init)(FN(state) *st)
 {
     const uint32_t K = st->K;
     const size_t P = st->P;
     #pragma omp parallel for schedule(static)
     for (int64_t i = 0; i < (int64_t)P; ++i) {
-        REAL sum = st->x[i];
-        for (uint32_t k = 1; k < K; ++k) sum = sum + st->x[(size_t)k * P + i];
-        st->xg[i] = sum / (REAL)K;
+        st->xg[i] = sum_over_workers(st, (size_t)i) / (REAL)K;
         st->u[i] = (REAL)0;
     }
     for (uint32_t k = 0; k < K; ++k) {
@@ -280,17 +298,7 @@ void FN(outer_sync)(FN(state) *st)
     const REAL oeps = (REAL)st->outer_eps;
     #pragma omp parallel for schedule(static)
     for (int64_t i = 0; i < (int64_t)P; ++i) {
-        REAL sum = st->x[i];
-        if (st->sum_groups > 1) {                        /* per machine first, then across machines */
-            const uint32_t per = K / st->sum_groups;
-            for (uint32_t gi = 0; gi < st->sum_groups; ++gi) {
-                REAL part = st->x[(size_t)(gi * per) * P + i];
-                for (uint32_t k = gi * per + 1; k < (gi + 1) * per; ++k) part = part + st->x[(size_t)k * P + i];
-                sum = gi == 0 ? part : sum + part;
-            }
-        } else {
-            for (uint32_t k = 1; k < K; ++k) sum = sum + st->x[(size_t)k * P + i];
-        }
+        REAL sum = sum_over_workers(st, (size_t)i);
         REAL xbar  = sum / (REAL)K;
         REAL delta = st->xg[i] - xbar;
         if (st->outer_opt == 1) {

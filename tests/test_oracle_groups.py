@@ -75,3 +75,18 @@ def test_uneven_groups_are_rejected():
     o = oracle.Oracle(np.zeros((6, 4), dtype=np.float32), K=6, H=1, p=0.0)
     with pytest.raises(ValueError):
         o.set_sum_groups(4)
+
+
+def test_initial_global_model_uses_the_same_two_level_sum():
+    rng = np.random.default_rng(11)
+    x0 = (rng.standard_normal((6, 500)) * 0.02).astype(np.float32)
+    plain = oracle.Oracle(x0, K=6, H=1, p=0.0)
+    two = oracle.Oracle(x0, K=6, H=1, p=0.0, sum_groups=2)
+    six = oracle.Oracle(x0, K=6, H=1, p=0.0, sum_groups=6)
+    assert np.array_equal(six.xg, plain.xg)                          # K groups of one worker: the plain sum
+    f = np.float32
+    want = (((x0[0] + x0[1]) + x0[2]) + ((x0[3] + x0[4]) + x0[5])) / f(6)      # numpy's binary32 operations
+    assert np.array_equal(two.xg, want)
+    assert not np.array_equal(two.xg, plain.xg) and np.max(np.abs(two.xg - plain.xg)) < 1e-8
+    exact = np.array([float(sum(Fraction(float(v)) for v in x0[:, i]) / 6) for i in range(500)])
+    assert np.max(np.abs(two.xg.astype(np.float64) - exact)) <= 8 * 2.0 ** -24 * np.max(np.abs(x0))
