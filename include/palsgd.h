@@ -213,6 +213,10 @@ int palsgd_outer_sync(palsgd_ctx* ctx, void* stream);
  * palsgd_outer_finish counts as the outer sync: n_outer += 1.
  * palsgd_set_worker_offset(k0) makes the local workers draw their decisions as workers
  * k0 .. k0+K_local-1 of the job (Algorithm 1's worker index); default 0.
+ * Initialisation: palsgd_init sets x_g to the mean of the LOCAL slots.  For the job's global
+ * model (the mean over all K_total workers, Sec. 2.2) run, once after palsgd_init on every GPU:
+ * palsgd_outer_partial -> the same all-reduce -> palsgd_global_from_exchange, which writes
+ * x_g = exchange / K_total and touches nothing else.
  * Errors: EINVAL (NULL, K_total < K_local, k0 + K_local > 2^32); EALIGN; EUNSUPPORTED (an
  * OUTER_SUB_ELEMS value whose stage does not fit in shared memory); ECUDA.
  */
@@ -220,6 +224,7 @@ int palsgd_exchange_numel(palsgd_ctx* ctx, uint64_t* n_floats);
 int palsgd_set_worker_offset(palsgd_ctx* ctx, uint32_t k0);
 int palsgd_outer_partial(palsgd_ctx* ctx, float* exchange, void* stream);
 int palsgd_outer_finish(palsgd_ctx* ctx, const float* exchange, uint32_t K_total, void* stream);
+int palsgd_global_from_exchange(palsgd_ctx* ctx, const float* exchange, uint32_t K_total, void* stream);
 
 /* The outer learning rate of the following outer syncs (it may follow a schedule, e.g. the
  * warm-up + cosine annealing of Appendix B: see palsgd_schedule_value).  Errors: EINVAL. */

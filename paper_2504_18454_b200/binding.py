@@ -86,7 +86,9 @@ def lib() -> C.CDLL:
     L.palsgd_set_worker_offset.argtypes = [vp, C.c_uint32]
     L.palsgd_outer_partial.argtypes = [vp, vp, vp]
     L.palsgd_outer_finish.argtypes = [vp, vp, C.c_uint32, vp]
-    for name in ("palsgd_exchange_numel", "palsgd_set_worker_offset", "palsgd_outer_partial", "palsgd_outer_finish"):
+    L.palsgd_global_from_exchange.argtypes = [vp, vp, C.c_uint32, vp]
+    for name in ("palsgd_exchange_numel", "palsgd_set_worker_offset", "palsgd_outer_partial", "palsgd_outer_finish",
+                 "palsgd_global_from_exchange"):
         getattr(L, name).restype = C.c_int
     L.palsgd_get_layout.argtypes = [vp, u64p, u64p, C.POINTER(C.c_uint32)]
     L.palsgd_get_layout.restype = C.c_int
@@ -292,6 +294,10 @@ class Palsgd:
     def outer_finish(self, exchange_ptr: int, K_total: int, stream: int = 0) -> None:
         self._check(lib().palsgd_outer_finish(self._ctx, C.c_void_p(exchange_ptr), int(K_total), C.c_void_p(stream)),
                     "palsgd_outer_finish")
+
+    def global_from_exchange(self, exchange_ptr: int, K_total: int, stream: int = 0) -> None:
+        self._check(lib().palsgd_global_from_exchange(self._ctx, C.c_void_p(exchange_ptr), int(K_total),
+                                                      C.c_void_p(stream)), "palsgd_global_from_exchange")
 
     def get_layout(self):
         ns, nc, ce = C.c_uint64(0), C.c_uint64(0), C.c_uint32(0)

@@ -715,6 +715,21 @@ extern "C" int palsgd_outer_partial(palsgd_ctx* ctx, float* exchange, void* stre
     return launch_checked(ctx, [&] { palsgd_outer_partial_kernel<8><<<grid, kThreads, 0, s>>>(a); });
 }
 
+extern "C" int palsgd_global_from_exchange(palsgd_ctx* ctx, const float* exchange, uint32_t K_total, void* stream)
+{
+    PALSGD_USABLE(ctx);
+    if (K_total < ctx->cfg.K) return PALSGD_EINVAL;
+    if (!exchange && ctx->exch_numel > 0) return PALSGD_EINVAL;
+    if (!aligned(exchange, 16)) return PALSGD_EALIGN;
+    if (ctx->n_oitems == 0) return PALSGD_OK;
+    OuterArgs a = outer_args(ctx);
+    a.sum_in = exchange;
+    a.Kf = (float)K_total;
+    const unsigned grid = grid_for(a.n_items, ctx->grid_cap_outer);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    return launch_checked(ctx, [&] { palsgd_global_from_sum_kernel<0><<<grid, kThreads, 0, s>>>(a); });
+}
+
 extern "C" int palsgd_outer_finish(palsgd_ctx* ctx, const float* exchange, uint32_t K_total, void* stream)
 {
     PALSGD_USABLE(ctx);

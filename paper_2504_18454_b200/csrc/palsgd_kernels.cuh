@@ -763,6 +763,22 @@ palsgd_outer_partial_kernel(const __grid_constant__ OuterArgs a)
     }
 }
 
+// Initialisation when the workers are spread over several GPUs: x_g = (sum over ALL workers) / K_total,
+// the sum having been formed by palsgd_outer_partial_kernel on every GPU and all-reduced.
+template <int UNUSED = 0>
+__global__ void __launch_bounds__(kThreads)
+palsgd_global_from_sum_kernel(const __grid_constant__ OuterArgs a)
+{
+    const Tables& tb = a.tb;
+    for (uint32_t item = blockIdx.x; item < a.n_items; item += gridDim.x) {
+        const Chunk ch = a.items[item];
+        const uint32_t seg = ch.seg & ~kSegVecFlag;
+        const float* sum = a.sum_in + tb.exch_off[seg] + ch.off;
+        float* xg = tb.global[seg] + ch.off;
+        for (uint32_t i = threadIdx.x; i < ch.len; i += kThreads) xg[i] = __fdiv_rn(sum[i], a.Kf);
+    }
+}
+
 // ---------------------------------------------------------------- DDP warm-up step
 // Mini-batch phase that precedes Algorithm 1 (Sec. 3.3, Sec. 4.1): per element the K
 // gradients are summed in ascending k and divided by K, ONE optimizer step is taken on

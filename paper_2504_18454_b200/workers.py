@@ -7,7 +7,8 @@ GPU holding all K workers would draw.  Every H steps the outer synchronisation r
 
     palsgd_outer_partial  ->  all-reduce(sum) of the exchange buffer  ->  palsgd_outer_finish
 
-(Algorithm 1's All-Reduce of the outer gradient, an average by Sec. 2.2; Eq. (3), Eq. (4)).
+(Algorithm 1's All-Reduce of the outer gradient, an average by Sec. 2.2; Eq. (3), Eq. (4)); the
+initial global model is formed the same way once (`init_global`).
 The all-reduce is `torch.distributed`'s (NCCL over NVLink between GPUs); this module is only
 the controller: which worker indices a rank owns, when to synchronise, and the three calls.
 It holds no arithmetic of the method.
@@ -55,6 +56,13 @@ class DistributedPalsgd:
                 if world > 1:
                     dist.all_reduce(buf, op=dist.ReduceOp.SUM)
         self._all_reduce = all_reduce_sum
+
+    def init_global(self, stream: int = 0) -> None:
+        """Once after the contexts have been created on every rank: the global model becomes the mean over
+        ALL workers of the job (palsgd_init alone gives every rank the mean of its own workers)."""
+        self.ctx.outer_partial(self.exchange.data_ptr(), stream)
+        self._all_reduce(self.exchange)
+        self.ctx.global_from_exchange(self.exchange.data_ptr(), self.K_total, stream)
 
     def inner_step(self, lr_t: float, eta_t: float, stream: int = 0) -> None:
         self.ctx.inner_step(lr_t, eta_t, stream)

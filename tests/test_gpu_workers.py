@@ -42,6 +42,8 @@ def test_one_rank_is_bit_identical_to_the_plain_outer_sync(layout, precision, ou
     exch = torch.zeros(split.lib.exchange_numel(), dtype=torch.float32, device=split.dev)
     assert exch.numel() >= P
     job = DistributedPalsgd(split.lib, exch, cfg.K, 0, 1, all_reduce_sum=lambda buf: None)
+    job.init_global(split.stream)                              # one rank: the mean palsgd_init formed, bit for bit
+    assert np.array_equal(split.state()["xg"], plain.state()["xg"])
     for t in range(cfg.T):
         g = _grads(cfg, P, t, cfg.K)
         plain.set_grads(g); split.set_grads(g)
@@ -55,18 +57,28 @@ def test_one_rank_is_bit_identical_to_the_plain_outer_sync(layout, precision, ou
 
 
 @pytest.mark.parametrize("inner,precision", [(0, 0), (1, 0), (0, 1)])
-def test_two_ranks_with_half_of_the_workers_each_match_one_oracle_with_all(inner, precision):
+def test_two_ranks_with_half_of_the_workers_each_match_the_oracle_bit_for_bit(inner, precision):
     K_total, world = 6, 2
     cfg = _cfg(K=K_total, inner=inner, precision=precision, momentum=0.9 if inner else 0.0, p=0.35)
     P = sum(RAGGED)
-    x_init = (np.random.default_rng(9).standard_normal(P) * 0.02).astype(np.float32)
-    x0 = np.tile(x_init, (K_total, 1))
-    orc = make_oracle(cfg, x0)
+    x0 = (np.random.default_rng(9).standard_normal((K_total, P)) * 0.02).astype(np.float32)   # workers start apart
+    from _harness import cfg_kwargs
+    import oracle
+    orc = oracle.Oracle(x0, sum_groups=world, **cfg_kwargs(cfg))     # sums per rank first, then across the two ranks
     local = cfg.with_(K=K_total // world)
-    ranks = [GpuRun(local, x0[: local.K], numel=RAGGED, layout="separate" if r else "arena") for r in range(world)]
+    ranks = [GpuRun(local, x0[r * local.K:(r + 1) * local.K], numel=RAGGED, layout="separate" if r else "arena")
+             for r in range(world)]
     for r, run in enumerate(ranks):
         run.lib.set_worker_offset(r * local.K)
     exch = [torch.zeros(run.lib.exchange_numel(), dtype=torch.float32, device=run.dev) for run in ranks]
+    # the job's initial global model: the mean over all workers, formed through the same exchange
+    for run, e in zip(ranks, exch):
+        run.lib.outer_partial(e.data_ptr(), run.stream)
+    total = exch[0] + exch[1]
+    for run, e in zip(ranks, exch):
+        e.copy_(total)
+        run.lib.global_from_exchange(e.data_ptr(), K_total, run.stream)
+        assert np.array_equal(run.state()["xg"], orc.xg)
     for t in range(cfg.T):
         g = _grads(cfg, P, t, K_total)
         orc.step(g, cfg.lr, cfg.eta)
@@ -89,12 +101,14 @@ def test_two_ranks_with_half_of_the_workers_each_match_one_oracle_with_all(inner
     for r, (run, st) in enumerate(zip(ranks, states)):
         sl = slice(r * local.K, (r + 1) * local.K)
         assert run.counters()["s"] == [int(v) for v in orc.s[sl]]
-        # grouped by rank, the sum over k rounds differently from the oracle's ascending order:
-        # the parity bar (1e-6 relative, 1e-7 absolute floor) applies, not bitwise equality
+
         class View:                                             # the oracle's rows of this rank
             dtype = orc.dtype
-            x, m, v, xg, u, uv, xw = orc.x[sl], orc.m[sl], orc.v[sl], orc.xg, orc.u, None, None
-        compare_state({k: v for k, v in st.items() if k != "xw"}, View)
+            x, m, v, xg, u, uv = orc.x[sl], orc.m[sl], orc.v[sl], orc.xg, orc.u, None
+            xw = orc.xw[sl] if orc.xw is not None else None
+        # the oracle adds the two ranks' partial sums exactly as the exchange does (two groups), so the
+        # comparison is bit for bit; against the one-level ascending sum only the parity bar would hold
+        compare_state(st, View, exact=True)
         assert run.guards_intact()
 
 
@@ -103,7 +117,9 @@ def test_argument_checks():
     run = GpuRun(cfg, np.zeros((cfg.K, 100), dtype=np.float32), numel=[100])
     buf = torch.zeros(run.lib.exchange_numel() + 4, dtype=torch.float32, device=run.dev)
     for call in (lambda: run.lib.outer_partial(0, run.stream), lambda: run.lib.outer_finish(0, cfg.K, run.stream),
-                 lambda: run.lib.outer_finish(buf.data_ptr(), cfg.K - 1, run.stream)):
+                 lambda: run.lib.outer_finish(buf.data_ptr(), cfg.K - 1, run.stream),
+                 lambda: run.lib.global_from_exchange(0, cfg.K, run.stream),
+                 lambda: run.lib.global_from_exchange(buf.data_ptr(), cfg.K - 1, run.stream)):
         with pytest.raises(Exception) as e:
             call()
         assert getattr(e.value, "status", None) == -1

@@ -41,14 +41,14 @@ dist.init_process_group("gloo")
 rank, world = dist.get_rank(), dist.get_world_size()
 K_total, P, H, T, p, seed = 4, 3001, 3, 7, 0.4, 77
 lr, eta = 1e-3, 16.0
-x_init = W.init_params_host(W.flat_shape(P), 1234, 0.02)
+x_all = np.stack([W.init_params_host(W.flat_shape(P), 1234 + k, 0.02) for k in range(K_total)])    # workers start apart
 
 
 class OracleContext:
     """Stands in for a device context: same methods, the oracle's arithmetic."""
-    def __init__(self, K, exchange):
+    def __init__(self, K, exchange, k_first):
         self.K, self.H, self.exchange, self.k0 = K, H, exchange, None
-        self.orc = oracle.Oracle(np.tile(x_init, (K, 1)), K=K, H=10**9, p=p, seed=seed)
+        self.orc = oracle.Oracle(x_all[k_first:k_first + K], K=K, H=10**9, p=p, seed=seed)
         self.calls = []
     def exchange_numel(self):
         return P
@@ -67,6 +67,9 @@ class OracleContext:
             acc = acc + self.orc.x[k]                       # float32, ascending local index
         self.exchange.copy_(torch.from_numpy(acc))
         self.calls.append("partial")
+    def global_from_exchange(self, ptr, K_tot, stream=0):
+        self.orc.xg[:] = (self.exchange.numpy() / np.float32(K_tot)).astype(np.float32)
+        self.calls.append("global")
     def outer_finish(self, ptr, K_tot, stream=0):
         xbar = (self.exchange.numpy() / np.float32(K_tot)).astype(np.float32)
         one = oracle.Oracle(xbar[None], K=1, H=1, p=0.0)    # OuterOPT on a one-worker average = xbar
@@ -79,12 +82,17 @@ class OracleContext:
 
 k0, k1 = worker_span(K_total, rank, world)
 exch = torch.zeros(P, dtype=torch.float32)
-ctx = OracleContext(k1 - k0, exch)
+ctx = OracleContext(k1 - k0, exch, k0)
 job = DistributedPalsgd(ctx, exch, K_total, rank, world)
+job.init_global()
 synced = [job.step(lr, eta) for _ in range(T)]
 
 # one oracle with all the workers, ascending order over all k
-ref = oracle.Oracle(np.tile(x_init, (K_total, 1)), K=K_total, H=H, p=p, seed=seed)
+ref = oracle.Oracle(x_all, K=K_total, H=H, p=p, seed=seed)
+grouped = oracle.Oracle(x_all, K=K_total, H=H, p=p, seed=seed, sum_groups=world)   # sums as the two ranks form them
+for t in range(T):
+    g = np.stack([W.grads_host(P, 5678, t, k, 0.01) for k in range(K_total)])
+    grouped.step(g, lr, eta)
 for t in range(T):
     g = np.stack([W.grads_host(P, 5678, t, k, 0.01) for k in range(K_total)])
     ref.step(g, lr, eta)
@@ -97,7 +105,9 @@ out = {"rank": rank, "k0": ctx.k0, "synced": synced, "calls": ctx.calls,
        "s_equal": [int(v) for v in ctx.orc.s] == [int(v) for v in ref.s[k0:k1]],
        "err_xg": err(ctx.orc.xg, ref.xg), "err_u": err(ctx.orc.u, ref.u),
        "err_x": err(ctx.orc.x, ref.x[k0:k1]), "m_equal": bool(np.array_equal(ctx.orc.m, ref.m[k0:k1])),
-       "n_pulls": int(sum(T - int(v) for v in ref.s))}
+       "n_pulls": int(sum(T - int(v) for v in ref.s)),
+       "bitwise_vs_grouped": bool(np.array_equal(ctx.orc.xg, grouped.xg) and np.array_equal(ctx.orc.u, grouped.u)
+                                  and np.array_equal(ctx.orc.x, grouped.x[k0:k1]))}
 with open(os.path.join(sys.argv[2], f"rank{rank}.json"), "w") as f:
     json.dump(out, f)
 dist.barrier()
@@ -117,8 +127,9 @@ def test_two_ranks_hold_half_of_the_workers_each(tmp_path):
         d = json.load(open(tmp_path / f"rank{rank}.json"))
         assert d["k0"] == 2 * rank
         assert d["synced"] == [False, False, True, False, False, True, False]       # H = 3, T = 7
-        assert d["calls"] == ["inner"] * 3 + ["partial", "finish"] + ["inner"] * 3 + ["partial", "finish"] + ["inner"]
-        assert d["same_xg_on_all_ranks"] and d["s_equal"] and d["m_equal"]
+        assert d["calls"] == (["partial", "global"] + ["inner"] * 3 + ["partial", "finish"] + ["inner"] * 3 +
+                              ["partial", "finish"] + ["inner"])
+        assert d["same_xg_on_all_ranks"] and d["s_equal"] and d["m_equal"] and d["bitwise_vs_grouped"]
         assert 0 < d["n_pulls"] < 4 * 7                                           # both branches were taken
         for key in ("err_xg", "err_u", "err_x"):                                  # the parity bar: 1e-6 rel, 1e-7 abs floor
             assert d[key] <= 1e-6, (key, d[key])
