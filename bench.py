@@ -484,6 +484,28 @@ def run_ours(args, cfg):
         ddp_ms = sum(evs[i].elapsed_time(evs[i + 1]) for i in range(8))
         ddp = {"ms": ddp_ms, "bytes": 8 * ddp_bytes_per_param(cfg) * Pn, "launches": 8}
 
+    # ---- the outer sync split around an exchange buffer (the form for workers spread over several GPUs;
+    # here one GPU, so the all-reduce between the two kernels is empty), timed on its own
+    split = None
+    if not args.no_ddp and world == 1:
+        exch = torch.zeros(ctx.exchange_numel(), dtype=torch.float32, device=dev)
+        pe, fe = [], []
+        for i in range(5):
+            for _ in range(2):
+                ctx.inner_step(cfg.lr, cfg.eta, stream)
+            e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+            e0.record(); ctx.outer_partial(exch.data_ptr(), stream)
+            e1.record(); ctx.outer_finish(exch.data_ptr(), K, stream)
+            e2.record()
+            if i > 0:
+                pe.append((e0, e1)); fe.append((e1, e2))
+        torch.cuda.synchronize(dev)
+        split = {"n": len(pe), "partial_ms": sum(a.elapsed_time(b) for a, b in pe),
+                 "finish_ms": sum(a.elapsed_time(b) for a, b in fe),
+                 "partial_bytes": len(pe) * (4 * K + 4) * Pn,
+                 "finish_bytes": len(fe) * ((6 if cfg.precision == 1 else 4) * K + 20) * Pn}
+        del exch
+
     # ---- the same two kernels on a ragged device layout (one allocation per worker and tensor), timed on their
     # own after the main regions: frameworks hold their parameters that way, and the packed arenas above are
     # the friendliest case for the multi-tensor metadata
@@ -565,6 +587,15 @@ def run_ours(args, cfg):
                                "note": "the same kernels over one allocation per (buffer kind, worker, tensor); "
                                        "timed on their own after the main regions; not part of value"}
                               if ragged else None),
+            "outer_split": ({"partial": roofline_entry("palsgd_outer_partial_kernel", "outer", cfg, peak, peak_src,
+                                                       split["partial_ms"], split["partial_bytes"], split["n"],
+                                                       traffic=None),
+                             "finish": roofline_entry("palsgd_outer_kernel (sum from the exchange buffer)", "outer", cfg,
+                                                      peak, peak_src, split["finish_ms"], split["finish_bytes"],
+                                                      split["n"], traffic=None),
+                             "note": "outer sync as local sum -> (all-reduce) -> finish, the form for workers spread "
+                                     "over several GPUs; one GPU here, no collective; not part of value"}
+                            if split else None),
             "graph_cycle": graph_cycle,
             "cpu_baseline": cpu_baseline,
             "e2e": ({"value": K * P_job * e2e["steps"] / (e2e["ms"] * 1e-3), "unit": UNIT,
