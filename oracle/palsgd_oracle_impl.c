@@ -361,10 +361,21 @@ void FN(ddp_step)(FN(state) *st, const void *grads, double alpha_t)
     if (!gbar) return;
     #pragma omp parallel for schedule(static)
     for (int64_t i = 0; i < (int64_t)P; ++i) {
-        REAL sum = g32 ? (REAL)g32[i] : (REAL)palsgd_oracle_bf16_to_f32(g16[i]);
-        for (uint32_t k = 1; k < K; ++k)
-            sum = sum + (g32 ? (REAL)g32[(size_t)k * P + i]
-                             : (REAL)palsgd_oracle_bf16_to_f32(g16[(size_t)k * P + i]));
+        /* ascending k; with the workers on several machines (sum_groups > 1) per machine first, then
+         * across the machines -- the order in which a DDP all-reduce of per-machine sums adds them */
+        #define GRAD_AT(k) (g32 ? (REAL)g32[(size_t)(k) * P + i] : (REAL)palsgd_oracle_bf16_to_f32(g16[(size_t)(k) * P + i]))
+        REAL sum = GRAD_AT(0);
+        if (st->sum_groups > 1) {
+            const uint32_t per = K / st->sum_groups;
+            for (uint32_t gi = 0; gi < st->sum_groups; ++gi) {
+                REAL part = GRAD_AT(gi * per);
+                for (uint32_t k = gi * per + 1; k < (gi + 1) * per; ++k) part = part + GRAD_AT(k);
+                sum = gi == 0 ? part : sum + part;
+            }
+        } else {
+            for (uint32_t k = 1; k < K; ++k) sum = sum + GRAD_AT(k);
+        }
+        #undef GRAD_AT
         gbar[i] = sum / (REAL)K;
     }
     /* in this phase the clip applies to the averaged gradient */

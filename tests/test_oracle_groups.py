@@ -90,3 +90,38 @@ def test_initial_global_model_uses_the_same_two_level_sum():
     assert not np.array_equal(two.xg, plain.xg) and np.max(np.abs(two.xg - plain.xg)) < 1e-8
     exact = np.array([float(sum(Fraction(float(v)) for v in x0[:, i]) / 6) for i in range(500)])
     assert np.max(np.abs(two.xg.astype(np.float64) - exact)) <= 8 * 2.0 ** -24 * np.max(np.abs(x0))
+
+
+@pytest.mark.parametrize("precision", [0, 1])
+def test_ddp_step_sums_the_gradients_in_the_same_two_levels(precision):
+    import workloads as W
+    K, P = 6, 700
+    rng = np.random.default_rng(21)
+    x0 = np.tile((rng.standard_normal(P) * 0.02).astype(np.float32), (K, 1))
+    g = (rng.standard_normal((K, P)) * 0.01).astype(np.float32)
+    gin = W.bf16_bits_from_f32_host(g) if precision else g
+    gval = (gin.astype(np.uint32) << 16).view(np.float32) if precision else g        # the values the step sees
+    runs = {G: oracle.Oracle(x0, K=K, H=10**6, p=0.0, precision=precision, sum_groups=G) for G in (0, 1, 2, 3, 6)}
+    for o in runs.values():
+        o.ddp_step(gin, 1e-3)
+    for G in (1, 6):                                   # one group / one worker per group: the plain sum
+        for name in ("x", "m", "v", "xg"):
+            assert np.array_equal(getattr(runs[G], name), getattr(runs[0], name)), (G, name)
+    # first AdamW step from zero moments: m = (1 - beta1) * gbar, so m / (1 - beta1) recovers the averaged gradient
+    f = np.float32
+    for G in (2, 3):
+        per = K // G
+        parts = []
+        for gi in range(G):
+            part = gval[gi * per].copy()
+            for k in range(gi * per + 1, (gi + 1) * per):
+                part = part + gval[k]
+            parts.append(part)
+        tot = parts[0]
+        for part in parts[1:]:
+            tot = tot + part
+        gbar = tot / f(K)
+        assert np.array_equal(runs[G].m[0], f(1.0 - 0.9) * gbar)
+        assert np.max(np.abs(runs[G].m[0] - runs[0].m[0])) < 1e-9
+    exact = np.array([float(sum(Fraction(float(v)) for v in gval[:, i]) / K) for i in range(P)])
+    assert np.max(np.abs(runs[2].m[0].astype(np.float64) / 0.1 - exact)) <= 1e-8
