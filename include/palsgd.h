@@ -226,6 +226,22 @@ int palsgd_outer_partial(palsgd_ctx* ctx, float* exchange, void* stream);
 int palsgd_outer_finish(palsgd_ctx* ctx, const float* exchange, uint32_t K_total, void* stream);
 int palsgd_global_from_exchange(palsgd_ctx* ctx, const float* exchange, uint32_t K_total, void* stream);
 
+/*
+ * The DDP warm-up step (see palsgd_ddp_step; Sec. 3.3, Sec. 4.1) for workers spread over several GPUs,
+ * around the same exchange buffer and the caller's all-reduce:
+ *   1. palsgd_ddp_partial:  exchange[i] = g_0[i] + ... + g_{K_local-1}[i]   (that order; bf16 widened exactly)
+ *   2. all-reduce (sum) of the exchange buffers
+ *   3. palsgd_ddp_finish:   gbar = exchange[i] / K_total, then exactly palsgd_ddp_step's optimizer step on
+ *      local worker 0's state, written to the K_local slots and to x_g; s_k, t as in palsgd_ddp_step.
+ * All ranks hold the same model and state in this phase and receive the same sum, so they stay identical.
+ * With one GPU the result is bit-identical to palsgd_ddp_step.  Gradient clipping is not offered in this form
+ * (the norm would be that of a gradient living in the exchange buffer).
+ * Errors: EINVAL (NULL, K_total < K_local, bad rate); EALIGN; EUNSUPPORTED (clipping on, or DDP_VARIANT 1);
+ * ECUDA.
+ */
+int palsgd_ddp_partial(palsgd_ctx* ctx, float* exchange, void* stream);
+int palsgd_ddp_finish(palsgd_ctx* ctx, const float* exchange, uint32_t K_total, double lr_t, void* stream);
+
 /* The outer learning rate of the following outer syncs (it may follow a schedule, e.g. the
  * warm-up + cosine annealing of Appendix B: see palsgd_schedule_value).  Errors: EINVAL. */
 int palsgd_set_outer_lr(palsgd_ctx* ctx, double outer_lr);

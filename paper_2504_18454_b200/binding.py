@@ -87,8 +87,10 @@ def lib() -> C.CDLL:
     L.palsgd_outer_partial.argtypes = [vp, vp, vp]
     L.palsgd_outer_finish.argtypes = [vp, vp, C.c_uint32, vp]
     L.palsgd_global_from_exchange.argtypes = [vp, vp, C.c_uint32, vp]
+    L.palsgd_ddp_partial.argtypes = [vp, vp, vp]
+    L.palsgd_ddp_finish.argtypes = [vp, vp, C.c_uint32, C.c_double, vp]
     for name in ("palsgd_exchange_numel", "palsgd_set_worker_offset", "palsgd_outer_partial", "palsgd_outer_finish",
-                 "palsgd_global_from_exchange"):
+                 "palsgd_global_from_exchange", "palsgd_ddp_partial", "palsgd_ddp_finish"):
         getattr(L, name).restype = C.c_int
     L.palsgd_get_layout.argtypes = [vp, u64p, u64p, C.POINTER(C.c_uint32)]
     L.palsgd_get_layout.restype = C.c_int
@@ -294,6 +296,13 @@ class Palsgd:
     def outer_finish(self, exchange_ptr: int, K_total: int, stream: int = 0) -> None:
         self._check(lib().palsgd_outer_finish(self._ctx, C.c_void_p(exchange_ptr), int(K_total), C.c_void_p(stream)),
                     "palsgd_outer_finish")
+
+    def ddp_partial(self, exchange_ptr: int, stream: int = 0) -> None:
+        self._check(lib().palsgd_ddp_partial(self._ctx, C.c_void_p(exchange_ptr), C.c_void_p(stream)), "palsgd_ddp_partial")
+
+    def ddp_finish(self, exchange_ptr: int, K_total: int, lr_t: float, stream: int = 0) -> None:
+        self._check(lib().palsgd_ddp_finish(self._ctx, C.c_void_p(exchange_ptr), int(K_total), lr_t, C.c_void_p(stream)),
+                    "palsgd_ddp_finish")
 
     def global_from_exchange(self, exchange_ptr: int, K_total: int, stream: int = 0) -> None:
         self._check(lib().palsgd_global_from_exchange(self._ctx, C.c_void_p(exchange_ptr), int(K_total),

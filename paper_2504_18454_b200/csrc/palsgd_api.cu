@@ -572,10 +572,10 @@ extern "C" int palsgd_inner_step(palsgd_ctx* ctx, double lr_t, double eta_t, voi
     return PALSGD_OK;
 }
 
-extern "C" int palsgd_ddp_step(palsgd_ctx* ctx, double lr_t, void* stream)
+// One DDP warm-up step.  sum_in == nullptr: the K local gradients are averaged in the kernel; otherwise the
+// gradient sum over all K_total workers of the job is read from the exchange buffer.
+static int ddp_launch(palsgd_ctx* ctx, double lr_t, void* stream, const float* sum_in, uint32_t K_total)
 {
-    PALSGD_USABLE(ctx);
-    if (!finite_nonneg(lr_t)) return PALSGD_EINVAL;
     const palsgd_config& c = ctx->cfg;
     DdpArgs a{};
     a.tb = ctx->tb;
@@ -590,7 +590,8 @@ extern "C" int palsgd_ddp_step(palsgd_ctx* ctx, double lr_t, void* stream)
     a.decay = (float)(1.0 - lr_t * c.weight_decay);
     a.mu = (float)c.momentum;
     a.wd = (float)c.weight_decay;
-    a.Kf = (float)c.K;
+    a.Kf = (float)K_total;
+    a.sum_in = sum_in;
     a.items = ctx->d_ditems;
     a.n_items = ctx->n_ditems;
     a.sub_elems = ctx->ddp_sub_elems;
@@ -615,15 +616,56 @@ extern "C" int palsgd_ddp_step(palsgd_ctx* ctx, double lr_t, void* stream)
     const bool bcast = ctx->ddp_variant != 1 && (int)stage_bytes <= ctx->smem_optin - 4096;   // measured best
     using DdpKernel = void (*)(const DdpArgs);
     DdpKernel kernel;
-    if (bcast) kernel = adam ? (bf ? palsgd_ddp_kernel<0, 1, 1> : palsgd_ddp_kernel<0, 0, 1>)
-                             : (bf ? palsgd_ddp_kernel<1, 1, 1> : palsgd_ddp_kernel<1, 0, 1>);
-    else       kernel = adam ? (bf ? palsgd_ddp_kernel<0, 1, 0> : palsgd_ddp_kernel<0, 0, 0>)
-                             : (bf ? palsgd_ddp_kernel<1, 1, 0> : palsgd_ddp_kernel<1, 0, 0>);
+    if (sum_in) {
+        if (!bcast) return PALSGD_EUNSUPPORTED;               // the exchange form exists in the staged form only
+        kernel = adam ? (bf ? palsgd_ddp_kernel<0, 1, 1, 1> : palsgd_ddp_kernel<0, 0, 1, 1>)
+                      : (bf ? palsgd_ddp_kernel<1, 1, 1, 1> : palsgd_ddp_kernel<1, 0, 1, 1>);
+    } else if (bcast) kernel = adam ? (bf ? palsgd_ddp_kernel<0, 1, 1> : palsgd_ddp_kernel<0, 0, 1>)
+                                    : (bf ? palsgd_ddp_kernel<1, 1, 1> : palsgd_ddp_kernel<1, 0, 1>);
+    else              kernel = adam ? (bf ? palsgd_ddp_kernel<0, 1, 0> : palsgd_ddp_kernel<0, 0, 0>)
+                                    : (bf ? palsgd_ddp_kernel<1, 1, 0> : palsgd_ddp_kernel<1, 0, 0>);
     if (bcast) { rc = ensure_dyn_smem(ctx, reinterpret_cast<const void*>(kernel), stage_bytes); if (rc) return rc; }
     rc = launch_checked(ctx, [&] { kernel<<<grid, kThreads, bcast ? stage_bytes : 0, s>>>(a); });
     if (rc) return rc;
     ctx->t += 1;
     return PALSGD_OK;
+}
+
+extern "C" int palsgd_ddp_step(palsgd_ctx* ctx, double lr_t, void* stream)
+{
+    PALSGD_USABLE(ctx);
+    if (!finite_nonneg(lr_t)) return PALSGD_EINVAL;
+    return ddp_launch(ctx, lr_t, stream, nullptr, ctx->cfg.K);
+}
+
+extern "C" int palsgd_ddp_partial(palsgd_ctx* ctx, float* exchange, void* stream)
+{
+    PALSGD_USABLE(ctx);
+    if (!exchange && ctx->exch_numel > 0) return PALSGD_EINVAL;
+    if (!aligned(exchange, 16)) return PALSGD_EALIGN;
+    if (ctx->n_ditems == 0) return PALSGD_OK;
+    DdpArgs a{};
+    a.tb = ctx->tb;
+    a.items = ctx->d_ditems;
+    a.n_items = ctx->n_ditems;
+    a.sum_out = exchange;
+    const unsigned grid = grid_for(a.n_items, ctx->grid_cap_outer);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const bool bf = ctx->cfg.precision == PALSGD_PREC_BF16_MASTER;
+    return launch_checked(ctx, [&] {
+        if (bf) palsgd_ddp_partial_kernel<1><<<grid, kThreads, 0, s>>>(a);
+        else    palsgd_ddp_partial_kernel<0><<<grid, kThreads, 0, s>>>(a);
+    });
+}
+
+extern "C" int palsgd_ddp_finish(palsgd_ctx* ctx, const float* exchange, uint32_t K_total, double lr_t, void* stream)
+{
+    PALSGD_USABLE(ctx);
+    if (!finite_nonneg(lr_t) || K_total < ctx->cfg.K) return PALSGD_EINVAL;
+    if (!exchange) return PALSGD_EINVAL;
+    if (!aligned(exchange, 16)) return PALSGD_EALIGN;
+    if (ctx->max_grad_norm > 0.0) return PALSGD_EUNSUPPORTED;  // the norm of a gradient that lives in the exchange buffer
+    return ddp_launch(ctx, lr_t, stream, exchange, K_total);
 }
 
 extern "C" int palsgd_pseudo_sync(palsgd_ctx* ctx, uint64_t worker_mask, double beta, void* stream)

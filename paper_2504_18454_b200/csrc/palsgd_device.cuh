@@ -116,6 +116,8 @@ struct DdpArgs {
     uint32_t n_stage;      // stage buffers in dynamic shared memory: 2 for a persistent grid, else 1
     uint32_t clip_on;      // 1: scale the averaged gradient by DevState::clip[0]
     uint32_t dynamic;      // 1: a persistent grid takes work items from DevState::queue
+    const float* sum_in;   // SUMIN kernels: the exchange buffer holding the gradient sum over ALL workers
+    float*       sum_out;  // partial-sum kernel: the exchange buffer that receives the local workers' sum
 };
 
 // Gradient-norm pass of the global-norm clip.

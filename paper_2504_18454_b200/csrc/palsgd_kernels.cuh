@@ -763,6 +763,67 @@ palsgd_outer_partial_kernel(const __grid_constant__ OuterArgs a)
     }
 }
 
+// DDP warm-up phase with the workers spread over several GPUs, first half: the local workers' gradients
+// added up in ascending local index (bf16 gradients widened exactly) into the exchange buffer.
+template <int PREC, int B = 8>
+__global__ void __launch_bounds__(kThreads)
+palsgd_ddp_partial_kernel(const __grid_constant__ DdpArgs a)
+{
+    __shared__ const void* s_g[kMaxWorkers];
+    const Tables& tb = a.tb;
+    const uint32_t K = tb.K;
+    for (uint32_t item = blockIdx.x; item < a.n_items; item += gridDim.x) {
+        const Chunk ch = a.items[item];
+        const uint32_t seg = ch.seg & ~kSegVecFlag;
+        __syncthreads();
+        if (threadIdx.x < K) {
+            const size_t pi = (size_t)threadIdx.x * tb.n_seg + seg;
+            if (PREC) s_g[threadIdx.x] = static_cast<const __nv_bfloat16*>(tb.grad[pi]) + ch.off;
+            else      s_g[threadIdx.x] = static_cast<const float*>(tb.grad[pi]) + ch.off;
+        }
+        __syncthreads();
+        float* out = a.sum_out + tb.exch_off[seg] + ch.off;
+        uint32_t done = 0;
+        if (ch.seg & kSegVecFlag) {
+            const uint32_t n4 = ch.len >> 2;
+            for (uint32_t i = threadIdx.x; i < n4; i += kThreads) {
+                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                for (uint32_t k0 = 0; k0 < K; k0 += B) {
+                    float4 R[PREC ? 1 : B]; uint2 H[PREC ? B : 1];
+#pragma unroll
+                    for (int j = 0; j < B; ++j)
+                        if (k0 + j < K) {
+                            if (PREC) H[j] = __ldcs(static_cast<const uint2*>(s_g[k0 + j]) + i);
+                            else      R[j] = __ldcs(static_cast<const float4*>(s_g[k0 + j]) + i);
+                        }
+#pragma unroll
+                    for (int j = 0; j < B; ++j)
+                        if (k0 + j < K) {
+                            float4 r;
+                            if (PREC) { float f[4]; unpack4(H[j], f); r = make_float4(f[0], f[1], f[2], f[3]); }
+                            else      { r = R[j]; }
+                            if (k0 + j == 0) acc = r;
+                            else { acc.x = __fadd_rn(acc.x, r.x); acc.y = __fadd_rn(acc.y, r.y);
+                                   acc.z = __fadd_rn(acc.z, r.z); acc.w = __fadd_rn(acc.w, r.w); }
+                        }
+                }
+                if ((reinterpret_cast<uintptr_t>(out) & 15u) == 0) reinterpret_cast<float4*>(out)[i] = acc;
+                else { out[4 * i] = acc.x; out[4 * i + 1] = acc.y; out[4 * i + 2] = acc.z; out[4 * i + 3] = acc.w; }
+            }
+            done = n4 << 2;
+        }
+        for (uint32_t i = done + threadIdx.x; i < ch.len; i += kThreads) {
+            float sum = 0.f;
+            for (uint32_t k = 0; k < K; ++k) {
+                const float gk = PREC ? __bfloat162float(static_cast<const __nv_bfloat16*>(s_g[k])[i])
+                                      : static_cast<const float*>(s_g[k])[i];
+                sum = k == 0 ? gk : __fadd_rn(sum, gk);
+            }
+            out[i] = sum;
+        }
+    }
+}
+
 // Initialisation when the workers are spread over several GPUs: x_g = (sum over ALL workers) / K_total,
 // the sum having been formed by palsgd_outer_partial_kernel on every GPU and all-reduced.
 template <int UNUSED = 0>
@@ -789,7 +850,9 @@ palsgd_global_from_sum_kernel(const __grid_constant__ OuterArgs a)
 // BCAST = 1: the new x, m, v (and bf16 copy) of a work item are staged in dynamic shared memory
 // ((12 or 8) + 2 bytes per element, sub_elems elements per buffer) and written to the K slots and
 // to x_g by bulk asynchronous stores; 16-byte-aligned pieces only, the rest takes the register path.
-template <int INNER, int PREC, int BCAST>
+// SUMIN = 1: the gradient sum over ALL workers of a job comes ready-made from the exchange buffer
+// (palsgd_ddp_partial_kernel on every GPU, then the caller's all-reduce) and Kf is the job's worker count.
+template <int INNER, int PREC, int BCAST, int SUMIN = 0>
 __global__ void __launch_bounds__(kThreads)
 palsgd_ddp_kernel(const __grid_constant__ DdpArgs a)
 {
@@ -833,6 +896,7 @@ palsgd_ddp_kernel(const __grid_constant__ DdpArgs a)
         }
         __syncthreads();
         float* xg = tb.global[seg] + ch.off;
+        const float* sum_src = SUMIN ? a.sum_in + tb.exch_off[seg] + ch.off : nullptr;
         unsigned char* stage = ddp_stage + (BCAST ? (walk.n % a.n_stage) * stage_bytes : 0u);
         float* sx = reinterpret_cast<float*>(stage);
         float* sm = sx + a.sub_elems;
@@ -847,7 +911,14 @@ palsgd_ddp_kernel(const __grid_constant__ DdpArgs a)
                 float4 V = make_float4(0.f, 0.f, 0.f, 0.f);
                 if (INNER == 0) V = __ldcs(reinterpret_cast<const float4*>(s_v[0]) + i);
                 float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-                for (uint32_t k0 = 0; k0 < K; k0 += B) {
+                if (SUMIN) {
+                    if ((reinterpret_cast<uintptr_t>(sum_src) & 15u) == 0)
+                        acc = __ldcs(reinterpret_cast<const float4*>(sum_src) + i);
+                    else
+                        acc = make_float4(__ldcs(sum_src + 4 * i), __ldcs(sum_src + 4 * i + 1),
+                                          __ldcs(sum_src + 4 * i + 2), __ldcs(sum_src + 4 * i + 3));
+                }
+                for (uint32_t k0 = 0; !SUMIN && k0 < K; k0 += B) {
                     // bf16 gradients stay packed in registers until they are added (half the registers)
                     float4 R[PREC ? 1 : B]; uint2 H[PREC ? B : 1];
 #pragma unroll
@@ -915,8 +986,8 @@ palsgd_ddp_kernel(const __grid_constant__ DdpArgs a)
             }
         }
         for (uint32_t i = done + threadIdx.x; i < ch.len; i += kThreads) {
-            float sum = 0.f;
-            for (uint32_t k = 0; k < K; ++k) {
+            float sum = SUMIN ? sum_src[i] : 0.f;
+            for (uint32_t k = 0; !SUMIN && k < K; ++k) {
                 const float gk = PREC ? __bfloat162float(static_cast<const __nv_bfloat16*>(s_g[k])[i])
                                       : static_cast<const float*>(s_g[k])[i];
                 sum = k == 0 ? gk : __fadd_rn(sum, gk);

@@ -64,6 +64,14 @@ class DistributedPalsgd:
         self._all_reduce(self.exchange)
         self.ctx.global_from_exchange(self.exchange.data_ptr(), self.K_total, stream)
 
+    def ddp_step(self, lr_t: float, stream: int = 0) -> None:
+        """One step of the DDP warm-up phase for the whole job: the gradients of all workers are averaged
+        (local sums, all-reduce, division by K_total) and every rank takes the same optimizer step."""
+        self.ctx.ddp_partial(self.exchange.data_ptr(), stream)
+        self._all_reduce(self.exchange)
+        self.ctx.ddp_finish(self.exchange.data_ptr(), self.K_total, lr_t, stream)
+        self.t += 1
+
     def inner_step(self, lr_t: float, eta_t: float, stream: int = 0) -> None:
         self.ctx.inner_step(lr_t, eta_t, stream)
         self.t += 1

@@ -138,6 +138,8 @@ def test_later_entry_points_reject_a_null_context():
     assert L.palsgd_outer_partial(None, None, None) == -1
     assert L.palsgd_outer_finish(None, None, 1, None) == -1
     assert L.palsgd_global_from_exchange(None, None, 1, None) == -1
+    assert L.palsgd_ddp_partial(None, None, None) == -1
+    assert L.palsgd_ddp_finish(None, None, 1, 1e-3, None) == -1
 
 
 @pytest.mark.parametrize("over", [dict(outer_opt=2), dict(outer_opt=1),                      # AdamW outer without outer_v

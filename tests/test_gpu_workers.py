@@ -112,6 +112,90 @@ def test_two_ranks_with_half_of_the_workers_each_match_the_oracle_bit_for_bit(in
         assert run.guards_intact()
 
 
+@pytest.mark.parametrize("layout", ["arena", "separate", "misaligned"])
+@pytest.mark.parametrize("inner,precision", [(0, 0), (0, 1), (1, 0), (1, 1)])
+def test_one_rank_ddp_step_through_the_exchange_is_bit_identical_to_the_plain_one(layout, inner, precision):
+    cfg = _cfg(inner=inner, precision=precision, momentum=0.9 if inner else 0.0)
+    P = sum(RAGGED)
+    x0 = np.tile((np.random.default_rng(5).standard_normal(P) * 0.02).astype(np.float32), (cfg.K, 1))
+    plain, split, orc = (GpuRun(cfg, x0, numel=RAGGED, layout=layout), GpuRun(cfg, x0, numel=RAGGED, layout=layout),
+                         make_oracle(cfg, x0))
+    exch = torch.zeros(split.lib.exchange_numel(), dtype=torch.float32, device=split.dev)
+    job = DistributedPalsgd(split.lib, exch, cfg.K, 0, 1, all_reduce_sum=lambda buf: None)
+    for t in range(4):
+        g = _grads(cfg, P, t, cfg.K)
+        plain.set_grads(g); split.set_grads(g)
+        plain.ddp_step(cfg.lr); job.ddp_step(cfg.lr, split.stream); orc.ddp_step(g, cfg.lr)
+    a, b = plain.state(), split.state()
+    for key in a:
+        assert np.array_equal(a[key], b[key]), key
+    compare_state(b, orc, exact=True)
+    assert split.counters()["t"] == 4 and split.counters()["s"] == [4] * cfg.K and split.guards_intact()
+    for t in range(4, 4 + cfg.T):                                # and on into Algorithm 1 from that state
+        g = _grads(cfg, P, t, cfg.K)
+        split.set_grads(g); orc.step(g, cfg.lr, cfg.eta); job.step(cfg.lr, cfg.eta, split.stream)
+    compare_state(split.state(), orc, exact=True)
+
+
+@pytest.mark.parametrize("inner,precision", [(0, 0), (1, 0), (0, 1), (1, 1)])
+def test_two_ranks_ddp_warm_up_then_algorithm_1_match_the_oracle_bit_for_bit(inner, precision):
+    K_total, world, n_ddp = 6, 2, 3
+    cfg = _cfg(K=K_total, inner=inner, precision=precision, momentum=0.9 if inner else 0.0, p=0.35, T=6)
+    P = sum(RAGGED)
+    x0 = np.tile((np.random.default_rng(11).standard_normal(P) * 0.02).astype(np.float32), (K_total, 1))
+    from _harness import cfg_kwargs
+    import oracle
+    orc = oracle.Oracle(x0, sum_groups=world, **cfg_kwargs(cfg))
+    local = cfg.with_(K=K_total // world)
+    ranks = [GpuRun(local, x0[r * local.K:(r + 1) * local.K], numel=RAGGED, layout="misaligned" if r else "arena")
+             for r in range(world)]
+    exch = [torch.zeros(run.lib.exchange_numel(), dtype=torch.float32, device=run.dev) for run in ranks]
+
+    def exchange_sum():                                         # the all-reduce of two ranks: one addition
+        total = exch[0] + exch[1]
+        for e in exch:
+            e.copy_(total)
+
+    for r, run in enumerate(ranks):
+        run.lib.set_worker_offset(r * local.K)
+    for t in range(n_ddp):
+        g = _grads(cfg, P, t, K_total)
+        orc.ddp_step(g, cfg.lr)
+        for r, run in enumerate(ranks):
+            run.set_grads(g[r * local.K:(r + 1) * local.K])
+            run.lib.ddp_partial(exch[r].data_ptr(), run.stream)
+        exchange_sum()
+        for r, run in enumerate(ranks):
+            run.lib.ddp_finish(exch[r].data_ptr(), K_total, cfg.lr, run.stream)
+    states = [run.state() for run in ranks]
+    for key in ("x", "m", "xg"):                                # all ranks took the same step
+        assert np.array_equal(states[0][key], states[1][key]), key
+    assert np.array_equal(states[0]["xg"], orc.xg) and np.array_equal(states[0]["x"][0], orc.x[0])
+    for t in range(n_ddp, n_ddp + cfg.T):
+        g = _grads(cfg, P, t, K_total)
+        orc.step(g, cfg.lr, cfg.eta)
+        for r, run in enumerate(ranks):
+            run.set_grads(g[r * local.K:(r + 1) * local.K])
+            run.inner_step(cfg.lr, cfg.eta)
+        if (t + 1) % cfg.H == 0:
+            for r, run in enumerate(ranks):
+                run.lib.outer_partial(exch[r].data_ptr(), run.stream)
+            exchange_sum()
+            for r, run in enumerate(ranks):
+                run.lib.outer_finish(exch[r].data_ptr(), K_total, run.stream)
+    assert orc.n_outer >= 2
+    for r, run in enumerate(ranks):
+        sl = slice(r * local.K, (r + 1) * local.K)
+        assert run.counters()["s"] == [int(v) for v in orc.s[sl]] and run.counters()["t"] == orc.t
+
+        class View:
+            dtype = orc.dtype
+            x, m, v, xg, u, uv = orc.x[sl], orc.m[sl], orc.v[sl], orc.xg, orc.u, None
+            xw = orc.xw[sl] if orc.xw is not None else None
+        compare_state(run.state(), View, exact=True)
+        assert run.guards_intact()
+
+
 def test_argument_checks():
     cfg = _cfg()
     run = GpuRun(cfg, np.zeros((cfg.K, 100), dtype=np.float32), numel=[100])
@@ -126,4 +210,19 @@ def test_argument_checks():
     with pytest.raises(Exception) as e:
         run.lib.outer_partial(buf.data_ptr() + 4, run.stream)
     assert getattr(e.value, "status", None) == -2
-    assert run.counters()["n_outer"] == 0
+    for call in (lambda: run.lib.ddp_partial(0, run.stream), lambda: run.lib.ddp_finish(0, cfg.K, 1e-3, run.stream),
+                 lambda: run.lib.ddp_finish(buf.data_ptr(), cfg.K - 1, 1e-3, run.stream),
+                 lambda: run.lib.ddp_finish(buf.data_ptr(), cfg.K, float("nan"), run.stream)):
+        with pytest.raises(Exception) as e:
+            call()
+        assert getattr(e.value, "status", None) == -1
+    with pytest.raises(Exception) as e:
+        run.lib.ddp_partial(buf.data_ptr() + 4, run.stream)
+    assert getattr(e.value, "status", None) == -2
+    run.set_grad_clip(1.0)                                       # no clipped form of the split step
+    run.lib.ddp_partial(buf.data_ptr(), run.stream)
+    with pytest.raises(Exception) as e:
+        run.lib.ddp_finish(buf.data_ptr(), cfg.K, 1e-3, run.stream)
+    assert getattr(e.value, "status", None) == -6
+    c = run.counters()
+    assert c["n_outer"] == 0 and c["t"] == 0

@@ -46,9 +46,10 @@ x_all = np.stack([W.init_params_host(W.flat_shape(P), 1234 + k, 0.02) for k in r
 
 class OracleContext:
     """Stands in for a device context: same methods, the oracle's arithmetic."""
-    def __init__(self, K, exchange, k_first):
+    def __init__(self, K, exchange, k_first, x_start=None):
         self.K, self.H, self.exchange, self.k0 = K, H, exchange, None
-        self.orc = oracle.Oracle(x_all[k_first:k_first + K], K=K, H=10**9, p=p, seed=seed)
+        x_start = x_all if x_start is None else x_start
+        self.orc = oracle.Oracle(x_start[k_first:k_first + K], K=K, H=10**9, p=p, seed=seed)
         self.calls = []
     def exchange_numel(self):
         return P
@@ -60,6 +61,18 @@ class OracleContext:
         forced = [oracle.decision(seed, t, self.k0 + k, p) for k in range(self.K)]
         self.orc.inner_step(g, lr_t, eta_t, forced=forced)
         self.calls.append("inner")
+    def ddp_partial(self, ptr, stream=0):
+        assert ptr == self.exchange.data_ptr()
+        acc = W.grads_host(P, 5678, self.orc.t, self.k0, 0.01)
+        for k in range(1, self.K):
+            acc = acc + W.grads_host(P, 5678, self.orc.t, self.k0 + k, 0.01)   # float32, ascending local index
+        self.exchange.copy_(torch.from_numpy(acc))
+        self.calls.append("ddp_partial")
+    def ddp_finish(self, ptr, K_tot, lr_t, stream=0):
+        assert self.K == 2                                   # (gbar + gbar) / 2 is gbar exactly
+        gbar = (self.exchange.numpy() / np.float32(K_tot)).astype(np.float32)
+        self.orc.ddp_step(np.tile(gbar, (self.K, 1)), lr_t)
+        self.calls.append("ddp_finish")
     def outer_partial(self, ptr, stream=0):
         assert ptr == self.exchange.data_ptr()
         acc = self.orc.x[0].copy()
@@ -87,6 +100,18 @@ job = DistributedPalsgd(ctx, exch, K_total, rank, world)
 job.init_global()
 synced = [job.step(lr, eta) for _ in range(T)]
 
+# the DDP warm-up phase: all workers start from one model; every rank must take the step of the job's mean gradient
+x_same = np.tile(x_all[0], (K_total, 1))
+exch2 = torch.zeros(P, dtype=torch.float32)
+ctx2 = OracleContext(k1 - k0, exch2, k0, x_same)
+job2 = DistributedPalsgd(ctx2, exch2, K_total, rank, world)
+ddp_ref = oracle.Oracle(x_same, K=K_total, H=H, p=p, seed=seed, sum_groups=world)
+for t in range(2):
+    job2.ddp_step(lr)
+    ddp_ref.ddp_step(np.stack([W.grads_host(P, 5678, t, k, 0.01) for k in range(K_total)]), lr)
+ddp_ok = bool(job2.t == 2 and np.array_equal(ctx2.orc.x, ddp_ref.x[k0:k1]) and np.array_equal(ctx2.orc.m, ddp_ref.m[k0:k1])
+              and np.array_equal(ctx2.orc.xg, ddp_ref.xg) and not np.array_equal(ddp_ref.xg, x_all[0]))
+
 # one oracle with all the workers, ascending order over all k
 ref = oracle.Oracle(x_all, K=K_total, H=H, p=p, seed=seed)
 grouped = oracle.Oracle(x_all, K=K_total, H=H, p=p, seed=seed, sum_groups=world)   # sums as the two ranks form them
@@ -105,6 +130,7 @@ out = {"rank": rank, "k0": ctx.k0, "synced": synced, "calls": ctx.calls,
        "s_equal": [int(v) for v in ctx.orc.s] == [int(v) for v in ref.s[k0:k1]],
        "err_xg": err(ctx.orc.xg, ref.xg), "err_u": err(ctx.orc.u, ref.u),
        "err_x": err(ctx.orc.x, ref.x[k0:k1]), "m_equal": bool(np.array_equal(ctx.orc.m, ref.m[k0:k1])),
+       "ddp_ok": ddp_ok, "ddp_calls": ctx2.calls,
        "n_pulls": int(sum(T - int(v) for v in ref.s)),
        "bitwise_vs_grouped": bool(np.array_equal(ctx.orc.xg, grouped.xg) and np.array_equal(ctx.orc.u, grouped.u)
                                   and np.array_equal(ctx.orc.x, grouped.x[k0:k1]))}
@@ -130,6 +156,7 @@ def test_two_ranks_hold_half_of_the_workers_each(tmp_path):
         assert d["calls"] == (["partial", "global"] + ["inner"] * 3 + ["partial", "finish"] + ["inner"] * 3 +
                               ["partial", "finish"] + ["inner"])
         assert d["same_xg_on_all_ranks"] and d["s_equal"] and d["m_equal"] and d["bitwise_vs_grouped"]
+        assert d["ddp_ok"] and d["ddp_calls"] == ["ddp_partial", "ddp_finish"] * 2
         assert 0 < d["n_pulls"] < 4 * 7                                           # both branches were taken
         for key in ("err_xg", "err_u", "err_x"):                                  # the parity bar: 1e-6 rel, 1e-7 abs floor
             assert d[key] <= 1e-6, (key, d[key])
