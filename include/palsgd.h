@@ -30,7 +30,10 @@
  *     is 16-byte aligned take the 128-bit vector path; so do tensors whose
  *     buffers all become 16-byte aligned after the same small number of leading
  *     elements (a packed list at an odd offset), behind a scalar head of those
- *     elements; anything else takes a scalar path.  Results are identical.
+ *     elements (at most 255: the library prefers the count that puts every
+ *     buffer on a multiple of 256 elements' bytes (1024 for fp32, 512 for bf16),
+ *     where the kernels run at their full rate; allocate there if you can);
+ *     anything else takes a scalar path.  Results are identical.
  *   - Arguments are checked before anything is enqueued: an EINVAL / EALIGN call
  *     has changed nothing.  If a CUDA call fails in the middle of an entry point
  *     (PALSGD_ECUDA), the context is marked failed and every later call that

@@ -13,7 +13,8 @@ Three layouts of the same tensor list:
                 one segment per tensor (a ragged list: a partial chunk at the end
                 of every tensor, tensors far smaller than a chunk).
   "misaligned"  as "arena", shifted by one element, so that no buffer is 16-byte
-                aligned and the library takes its scalar path.
+                aligned: the library peels a scalar head off the front and runs
+                the rest on its vector path.
 
 This module only allocates, slices and copies: no arithmetic.
 """
@@ -68,7 +69,7 @@ class ReplicaArena:
                     per_row.append(row)
                 self._views[name] = per_row
         else:
-            Ppad = (self.P + self._shift + 63) // 64 * 64    # rows stay 128-byte aligned
+            Ppad = (self.P + self._shift + 255) // 256 * 256  # rows start on multiples of 256 elements (1024 bytes of fp32)
             for name, (rows, dt) in kinds.items():
                 a = torch.zeros((rows, Ppad), dtype=dt, device=self.device)
                 self.t[name] = a

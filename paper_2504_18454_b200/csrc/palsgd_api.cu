@@ -34,8 +34,8 @@ struct Segment {
     size_t   first_tensor;
     size_t   n_tensors;
     uint64_t numel;
-    int      head;     // elements to peel off the front so that what follows is 16-byte aligned in every
-                       // buffer (0..7); -1 = no such count exists: the whole segment takes the scalar path
+    int      head;     // elements to peel off the front so that what follows is aligned (16 bytes at least) in every
+                       // buffer (0..255); -1 = no such count exists: the whole segment takes the scalar path
 };
 
 struct palsgd_ctx {
@@ -386,21 +386,31 @@ extern "C" int palsgd_init(palsgd_ctx** out, const palsgd_config* cfg, size_t n_
         return ga + numel[j] * 4 == reinterpret_cast<const char*>(bufs->global[j + 1]) &&
                ua + numel[j] * 4 == reinterpret_cast<const char*>(bufs->outer_mom[j + 1]);
     };
-    // Elements to peel off a segment's front so that the rest is 16-byte aligned in every buffer: h with
-    // (address + h * element size) % 16 == 0 for all of them (0 for buffers that are aligned already,
-    // 7 for a packed list shifted by one element: fp32 at +4 bytes, bf16 at +2).  -1 if there is none.
+    // Elements to peel off a segment's front so that what follows is aligned in every buffer.  Needed
+    // by the vector paths and the bulk stores: 16 bytes.  Wanted: a multiple of 256 elements (1024
+    // bytes of fp32, 512 of bf16).  Measured on packed lists shifted by s elements: the inner kernel
+    // runs at its full rate for s = 256, 1.5 % under it for s = 128, 3-5 % under it for any s below
+    // that, 16-byte aligned or not.  So: the smallest h that puts every fp32 buffer on 1024 bytes and
+    // every bf16 buffer on 512, else on 512 and 256, else on 256 and 128, else all on 16: 0 for buffers
+    // that are aligned already, 255 for a packed list shifted by one element, 7 or less when the
+    // buffers' offsets differ.  -1 if no h gives even 16 bytes.
     auto head_of = [&](size_t first) {
-        for (int h = 0; h < 8; ++h) {
-            bool ok = aligned(reinterpret_cast<const char*>(bufs->global[first]) + 4 * h, 16) &&
-                      aligned(reinterpret_cast<const char*>(bufs->outer_mom[first]) + 4 * h, 16) &&
-                      (!oadam || aligned(reinterpret_cast<const char*>(bufs->outer_v[first]) + 4 * h, 16));
-            for (uint32_t k = 0; k < K && ok; ++k)
+        auto all_aligned = [&](int h, size_t a4, size_t a2) {    // bytes wanted: 4-byte kinds, 2-byte kinds
+            if (!aligned(reinterpret_cast<const char*>(bufs->global[first]) + 4 * h, a4) ||
+                !aligned(reinterpret_cast<const char*>(bufs->outer_mom[first]) + 4 * h, a4) ||
+                (oadam && !aligned(reinterpret_cast<const char*>(bufs->outer_v[first]) + 4 * h, a4)))
+                return false;
+            for (uint32_t k = 0; k < K; ++k)
                 for (const Kind& kd : kinds)
                     if (kd.present && !aligned(static_cast<const char*>(buf_ptr(bufs, kd.id, (size_t)k * n_tensors + first)) +
-                                                   kd.esize * h, 16))
-                        ok = false;
-            if (ok) return h;
-        }
+                                                   kd.esize * h, kd.esize == 4 ? a4 : a2))
+                        return false;
+            return true;
+        };
+        const size_t want[4][2] = {{1024, 512}, {512, 256}, {256, 128}, {16, 16}};
+        for (const auto& w : want)
+            for (int h = 0; h < (int)(w[1] / 2); ++h)
+                if (all_aligned(h, w[0], w[1])) return h;
         return -1;
     };
     for (size_t j = 0; j < n_tensors;) {

@@ -37,7 +37,7 @@ class GpuRun:
     """
 
     def __init__(self, cfg, x0: np.ndarray, numel: Optional[Sequence[int]] = None,
-                 layout: str = "arena", device: str = "cuda:0"):
+                 layout: str = "arena", device: str = "cuda:0", row_align: int = 8):
         self.cfg, self.layout, self.dev = cfg, layout, torch.device(device)
         self.numel = [int(n) for n in (numel if numel is not None else [t.numel for t in cfg.tensors])]
         self.K, self.Ptot = cfg.K, int(sum(self.numel))
@@ -57,7 +57,7 @@ class GpuRun:
             kinds["outer_v"] = (torch.float32, 1)
         self.arena: Dict[str, torch.Tensor] = {}
         self.views: Dict[str, List[List[torch.Tensor]]] = {}
-        row = (self.off + self.Ptot + GUARD + 8 + 7) // 8 * 8
+        row = (self.off + self.Ptot + GUARD + 8 + row_align - 1) // row_align * row_align   # elements per arena row
         for name, (dt, rows) in kinds.items():
             if layout == "separate":
                 self.views[name] = [[torch.full((n,), SENTINEL, dtype=dt, device=self.dev)

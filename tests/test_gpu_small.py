@@ -61,6 +61,30 @@ def test_ragged_tensor_list_matches_oracle(layout, inner, precision):
     _run_both(cfg, RAGGED, layout)
 
 
+@pytest.mark.parametrize("precision", [0, 1])
+@pytest.mark.parametrize("numel", [[50], [64, 3], [191], [190, 9], [8192 + 70, 5, 200]])
+def test_long_scalar_head_in_front_of_a_list_one_element_off_a_256_element_grid(numel, precision):
+    # rows a multiple of 256 elements apart: every buffer starts 64 + 1 elements behind a multiple of 256 elements, and
+    # the library peels the 191 elements that put all of them back on one (more than some of these lists hold) instead
+    # of the 3 or 7 that 16 bytes would need
+    cfg = _cfg(numel, K=3, H=3, T=7, precision=precision)
+    P = int(sum(numel))
+    x0 = _x0(cfg.K, P)
+    gpu, orc = GpuRun(cfg, x0, numel=numel, layout="misaligned", row_align=256), make_oracle(cfg, x0)
+    lay, head = gpu.lib.get_layout(), 191
+    assert lay["n_segments"] == 1 and lay["n_chunks"] == 1 + (0 if P <= head else -(-(P - head) // lay["chunk_elems"]))
+    gpu.set_grad_clip(0.05); orc.set_grad_clip(0.05)
+    for t in range(2):                                            # the DDP kernel and the norm pass over the same pieces
+        g = _grads(cfg, P, t)
+        gpu.set_grads(g); gpu.ddp_step(cfg.lr); orc.ddp_step(g, cfg.lr)
+    for t in range(2, 2 + cfg.T):
+        g = _grads(cfg, P, t)
+        gpu.set_grads(g); gpu.step(cfg.lr, cfg.eta); orc.step(g, cfg.lr, cfg.eta)
+        assert gpu.counters()["last_b"] == [int(v) for v in orc.last_b]
+    compare_state(gpu.state(), orc, exact=True)
+    assert gpu.counters()["n_outer"] == orc.n_outer >= 2 and gpu.guards_intact()
+
+
 @pytest.mark.parametrize("K", [1, 2, 3, 8, 32, 64])
 def test_worker_counts(K):
     numel = [4096 * 2 + 13]
@@ -297,7 +321,12 @@ def test_layout_report_counts_segments_and_chunks():
     # packed: the empty tensor (a NULL pointer) ends the first run of adjacent tensors
     packed = GpuRun(cfg, x0, numel=numel, layout="arena").lib.get_layout()
     assert packed == {"n_segments": 2, "n_chunks": 4, "chunk_elems": 8192}
-    shifted = GpuRun(cfg, x0, numel=numel, layout="misaligned").lib.get_layout()
-    assert shifted["n_segments"] == 2 and shifted["n_chunks"] == 6       # per segment a short scalar head, then aligned chunks
+    # one element off, rows a multiple of 256 elements apart: per segment a scalar head up to the next multiple of 256
+    # elements (191 and 179 of them), then aligned chunks: 1 + 2 and 1 + 0
+    shifted = GpuRun(cfg, x0, numel=numel, layout="misaligned", row_align=256).lib.get_layout()
+    assert shifted["n_segments"] == 2 and shifted["n_chunks"] == 4
+    # rows 8 elements (mod 128) apart: no common boundary beyond 16 bytes, heads of 3 elements: 1 + 3 and 1 + 1
+    shifted = GpuRun(cfg, _x0(cfg.K, sum(numel) + 8), numel=numel + [8], layout="misaligned").lib.get_layout()
+    assert shifted["n_segments"] == 2 and shifted["n_chunks"] == 6
     apart = GpuRun(cfg, x0, numel=numel, layout="separate").lib.get_layout()
     assert apart["n_segments"] == 3 and apart["n_chunks"] == 5
