@@ -37,7 +37,7 @@ class GpuRun:
     """
 
     def __init__(self, cfg, x0: np.ndarray, numel: Optional[Sequence[int]] = None,
-                 layout: str = "arena", device: str = "cuda:0", row_align: int = 8):
+                 layout: str = "arena", device: str = "cuda:0", row_align: int = 8, shift: int = 1):
         self.cfg, self.layout, self.dev = cfg, layout, torch.device(device)
         self.numel = [int(n) for n in (numel if numel is not None else [t.numel for t in cfg.tensors])]
         self.K, self.Ptot = cfg.K, int(sum(self.numel))
@@ -45,7 +45,7 @@ class GpuRun:
         self.bf = cfg.precision == 1
         self.adam = cfg.inner == 0
         pdt = torch.bfloat16 if self.bf else torch.float32
-        self.off = GUARD + (1 if layout == "misaligned" else 0)
+        self.off = GUARD + (shift if layout == "misaligned" else 0)   # "misaligned": every row starts `shift` elements late
         self.starts = np.concatenate([[0], np.cumsum(self.numel)]).astype(np.int64)
         kinds = {"param": (pdt, self.K), "grad": (pdt, self.K), "m": (torch.float32, self.K),
                  "global_": (torch.float32, 1), "outer_mom": (torch.float32, 1)}

@@ -44,17 +44,21 @@ def _case(seed):
         knobs[P.TUNE_DDP_VARIANT] = int(rng.choice([0, 1, 2]))
     n_ddp = int(rng.integers(0, 3))
     clip = float(rng.choice([0.0, 0.0, 0.05]))
-    return cfg, numel, layout, knobs, n_ddp, clip
+    # where the rows of a packed layout start: how far apart (elements) and how far off that grid; decides the
+    # scalar head the library peels (0 to 255 elements)
+    place = np.random.default_rng(5000 + seed)
+    geometry = dict(row_align=int(place.choice([8, 8, 64, 128, 256])), shift=int(place.choice([1, 1, 2, 3, 5, 100, 201])))
+    return cfg, numel, layout, knobs, n_ddp, clip, geometry
 
 
 @pytest.mark.parametrize("seed", range(160))
 def test_random_configuration_matches_the_oracle_bit_for_bit(seed):
-    cfg, numel, layout, knobs, n_ddp, clip = _case(seed)
+    cfg, numel, layout, knobs, n_ddp, clip, geometry = _case(seed)
     Pn = int(sum(numel))
     x0 = (np.random.default_rng(seed).standard_normal((cfg.K, Pn)) * 0.02).astype(np.float32)
     if n_ddp:
         x0 = np.tile(x0[0], (cfg.K, 1))                  # the warm-up phase starts from a common model
-    gpu, orc = GpuRun(cfg, x0, numel=numel, layout=layout), make_oracle(cfg, x0)
+    gpu, orc = GpuRun(cfg, x0, numel=numel, layout=layout, **geometry), make_oracle(cfg, x0)
     for knob, value in knobs.items():
         gpu.lib.set_tuning(knob, value)
     if clip:

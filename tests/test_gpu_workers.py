@@ -147,7 +147,7 @@ def test_two_ranks_ddp_warm_up_then_algorithm_1_match_the_oracle_bit_for_bit(inn
     import oracle
     orc = oracle.Oracle(x0, sum_groups=world, **cfg_kwargs(cfg))
     local = cfg.with_(K=K_total // world)
-    ranks = [GpuRun(local, x0[r * local.K:(r + 1) * local.K], numel=RAGGED, layout="misaligned" if r else "arena")
+    ranks = [GpuRun(local, x0[r * local.K:(r + 1) * local.K], numel=RAGGED, layout="misaligned" if r else "arena", row_align=256 if r else 8)
              for r in range(world)]
     exch = [torch.zeros(run.lib.exchange_numel(), dtype=torch.float32, device=run.dev) for run in ranks]
 
