@@ -499,11 +499,24 @@ def run_ours(args, cfg):
             e2.record()
             if i > 0:
                 pe.append((e0, e1)); fe.append((e1, e2))
+        dpe, dfe = [], []                                  # the DDP warm-up step, split the same way
+        g_es = 2 if cfg.precision == 1 else 4              # bytes per gradient element
+        for i in range(5):
+            e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+            e0.record(); ctx.ddp_partial(exch.data_ptr(), stream)
+            e1.record(); ctx.ddp_finish(exch.data_ptr(), K, cfg.lr, stream)
+            e2.record()
+            if i > 0:
+                dpe.append((e0, e1)); dfe.append((e1, e2))
         torch.cuda.synchronize(dev)
         split = {"n": len(pe), "partial_ms": sum(a.elapsed_time(b) for a, b in pe),
                  "finish_ms": sum(a.elapsed_time(b) for a, b in fe),
                  "partial_bytes": len(pe) * (4 * K + 4) * Pn,
-                 "finish_bytes": len(fe) * ((6 if cfg.precision == 1 else 4) * K + 20) * Pn}
+                 "finish_bytes": len(fe) * ((6 if cfg.precision == 1 else 4) * K + 20) * Pn,
+                 "ddp_partial_ms": sum(a.elapsed_time(b) for a, b in dpe),
+                 "ddp_finish_ms": sum(a.elapsed_time(b) for a, b in dfe),
+                 "ddp_partial_bytes": len(dpe) * (g_es * K + 4) * Pn,
+                 "ddp_finish_bytes": len(dfe) * (ddp_bytes_per_param(cfg) - g_es * K + 4) * Pn}
         del exch
 
     # ---- the same two kernels on a ragged device layout (one allocation per worker and tensor), timed on their
@@ -593,8 +606,15 @@ def run_ours(args, cfg):
                              "finish": roofline_entry("palsgd_outer_kernel (sum from the exchange buffer)", "outer", cfg,
                                                       peak, peak_src, split["finish_ms"], split["finish_bytes"],
                                                       split["n"], traffic=None),
-                             "note": "outer sync as local sum -> (all-reduce) -> finish, the form for workers spread "
-                                     "over several GPUs; one GPU here, no collective; not part of value"}
+                             "ddp_partial": roofline_entry("palsgd_ddp_partial_kernel", "ddp", cfg, peak, peak_src,
+                                                           split["ddp_partial_ms"], split["ddp_partial_bytes"],
+                                                           split["n"], traffic=None),
+                             "ddp_finish": roofline_entry("palsgd_ddp_kernel (gradient sum from the exchange buffer)",
+                                                          "ddp", cfg, peak, peak_src, split["ddp_finish_ms"],
+                                                          split["ddp_finish_bytes"], split["n"], traffic=None),
+                             "note": "outer sync and DDP warm-up step as local sum -> (all-reduce) -> finish, the form "
+                                     "for workers spread over several GPUs; one GPU here, no collective; not part of "
+                                     "value"}
                             if split else None),
             "graph_cycle": graph_cycle,
             "cpu_baseline": cpu_baseline,

@@ -653,11 +653,11 @@ extern "C" int palsgd_ddp_partial(palsgd_ctx* ctx, float* exchange, void* stream
     PALSGD_USABLE(ctx);
     if (!exchange && ctx->exch_numel > 0) return PALSGD_EINVAL;
     if (!aligned(exchange, 16)) return PALSGD_EALIGN;
-    if (ctx->n_ditems == 0) return PALSGD_OK;
+    if (ctx->tb.n_chunks == 0) return PALSGD_OK;
     DdpArgs a{};
     a.tb = ctx->tb;
-    a.items = ctx->d_ditems;
-    a.n_items = ctx->n_ditems;
+    a.items = ctx->tb.chunks;                               // nothing is staged: the inner kernel's larger pieces serve
+    a.n_items = ctx->tb.n_chunks;
     a.sum_out = exchange;
     const unsigned grid = grid_for(a.n_items, ctx->grid_cap_outer);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -759,9 +759,13 @@ extern "C" int palsgd_outer_partial(palsgd_ctx* ctx, float* exchange, void* stre
     PALSGD_USABLE(ctx);
     if (!exchange && ctx->exch_numel > 0) return PALSGD_EINVAL;
     if (!aligned(exchange, 16)) return PALSGD_EALIGN;
-    if (ctx->n_oitems == 0) return PALSGD_OK;
+    if (ctx->tb.n_chunks == 0) return PALSGD_OK;
     OuterArgs a = outer_args(ctx);
     a.sum_out = exchange;
+    // nothing is staged here, so the larger pieces of the inner kernel's chunk table serve: the per-item
+    // set-up (two barriers, K pointers) is paid once per 4096 or 8192 elements instead of once per 1024
+    a.items = ctx->tb.chunks;
+    a.n_items = ctx->tb.n_chunks;
     const unsigned grid = grid_for(a.n_items, ctx->grid_cap_outer);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     return launch_checked(ctx, [&] { palsgd_outer_partial_kernel<8><<<grid, kThreads, 0, s>>>(a); });

@@ -32,7 +32,8 @@ def test_bench_line_has_the_contract_keys():
     assert d["roofline"]["bound"] == "hbm" and d["roofline"]["achieved"] > 0 and d["gpu_launches"] == 16 + 2
     assert d["cpu_baseline"]["kind"] == "oracle" and d["e2e"]["h2d_bytes_per_step"] > 0
     assert d["config"]["workload"] == "c0_flat_1m" and d["value"] > 0
-    assert d["outer_split"]["partial"]["achieved"] > 0 and d["outer_split"]["finish"]["achieved"] > 0
+    for part in ("partial", "finish", "ddp_partial", "ddp_finish"):
+        assert d["outer_split"][part]["achieved"] > 0
 
 
 def test_outer_sync_is_timed_even_when_no_sync_falls_inside_the_step_loop():
