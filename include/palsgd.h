@@ -357,6 +357,21 @@ int palsgd_get_launch_count(palsgd_ctx* ctx, uint64_t* n_launches);
  * per worker each) and the chunk size.  Any output pointer may be NULL.  Errors: EINVAL. */
 int palsgd_get_layout(palsgd_ctx* ctx, uint64_t* n_segments, uint64_t* n_chunks, uint32_t* chunk_elems);
 
+/* The same report WITHOUT a context and without touching the GPU: what palsgd_init would make of this
+ * tensor list (the multi-tensor launch metadata of the path).  A pure host function of the configuration,
+ * the sizes and the ADDRESSES in `bufs` (same tables as for palsgd_init; nothing they point to is read,
+ * so it may be called before the buffers hold anything, or from a process without a GPU).
+ * Per segment i < *n_segments, if the array pointers are non-NULL (capacity: n_tensors entries each):
+ *   seg_first_tensor[i], seg_n_tensors[i]  the run of tensors fused into it (tensors adjacent in every buffer;
+ *                                          empty tensors inside a run are skipped over, an all-empty run is dropped)
+ *   seg_head[i]   leading elements handled by the scalar path so that the rest is aligned in every buffer
+ *                 (see the alignment rule above): 0..255, or -1 = the whole segment takes the scalar path
+ * Errors: exactly palsgd_init's argument errors (EINVAL, EALIGN); no other. */
+int palsgd_plan_layout(const palsgd_config* cfg, size_t n_tensors, const uint64_t* numel,
+                       const palsgd_buffers* bufs, uint64_t* n_segments, uint64_t* n_chunks,
+                       uint32_t* chunk_elems, uint64_t* seg_first_tensor, uint64_t* seg_n_tensors,
+                       int32_t* seg_head);
+
 /* Launch-shape knobs (advanced; results never depend on them).  Setting any of them drops a cycle recorded by
  * palsgd_cycle_capture (palsgd_cycle_launch then returns ESTATE until the cycle is captured again).
  * *_GRID_CAP: the largest grid a launch may use, CTAs looping over work items

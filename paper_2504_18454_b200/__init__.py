@@ -9,6 +9,7 @@ from .binding import (  # noqa: F401
     Palsgd,
     PalsgdError,
     decision,
+    plan_layout,
     schedule_value,
     OUTER_SGD,
     OUTER_ADAMW,

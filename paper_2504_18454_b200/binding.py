@@ -87,6 +87,9 @@ def lib() -> C.CDLL:
     L.palsgd_outer_partial.argtypes = [vp, vp, vp]
     L.palsgd_outer_finish.argtypes = [vp, vp, C.c_uint32, vp]
     L.palsgd_global_from_exchange.argtypes = [vp, vp, C.c_uint32, vp]
+    L.palsgd_plan_layout.argtypes = [C.POINTER(Config), C.c_size_t, u64p, C.POINTER(Buffers), u64p, u64p,
+                                     C.POINTER(C.c_uint32), u64p, u64p, C.POINTER(C.c_int32)]
+    L.palsgd_plan_layout.restype = C.c_int
     L.palsgd_ddp_partial.argtypes = [vp, vp, vp]
     L.palsgd_ddp_finish.argtypes = [vp, vp, C.c_uint32, C.c_double, vp]
     for name in ("palsgd_exchange_numel", "palsgd_set_worker_offset", "palsgd_outer_partial", "palsgd_outer_finish",
@@ -161,6 +164,34 @@ def outer_sync_noalloc(*, K: int, numel: Sequence[int], params, global_, outer_m
         float(outer_lr), float(outer_momentum), int(bool(outer_nesterov)), C.c_void_p(stream))
     if rc:
         raise PalsgdError(rc, "palsgd_outer_sync_noalloc")
+
+
+def plan_layout(*, K: int, numel: Sequence[int], param, grad, m, global_, outer_mom, v=None, master=None,
+                outer_v=None, inner: int = INNER_ADAMW, precision: int = PREC_FP32, outer_opt: int = OUTER_SGD):
+    """What palsgd_init would make of a tensor list, from ADDRESSES alone (plain integers; nothing is
+    dereferenced and no GPU is needed): param / grad / m / v / master are K rows of len(numel) addresses,
+    global_ / outer_mom / outer_v one row.  Returns the segment and chunk counts and, per segment,
+    (first tensor, tensors fused, scalar head)."""
+    n = len(numel)
+    cfg = Config(K=K, inner=inner, H=1, p=0.5, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.0, momentum=0.0,
+                 outer_lr=1.0, outer_momentum=0.0, outer_nesterov=0, precision=precision, seed=0,
+                 outer_opt=outer_opt, reserved_=0, outer_beta1=0.9, outer_beta2=0.999, outer_eps=1e-8,
+                 outer_weight_decay=0.0)
+    flat = lambda rows: _ptr_array([int(a) for row in rows for a in row])
+    arrs = {"param": flat(param), "grad": flat(grad), "m": flat(m),
+            "master": flat(master) if master is not None else None, "v": flat(v) if v is not None else None,
+            "global_": _ptr_array([int(a) for a in global_]), "outer_mom": _ptr_array([int(a) for a in outer_mom]),
+            "outer_v": _ptr_array([int(a) for a in outer_v]) if outer_v is not None else None}
+    bufs = Buffers(**{k: (C.cast(a, C.POINTER(C.c_void_p)) if a is not None else None) for k, a in arrs.items()})
+    nm = (C.c_uint64 * n)(*[int(x) for x in numel])
+    ns, nc, ce = C.c_uint64(0), C.c_uint64(0), C.c_uint32(0)
+    first, count, head = (C.c_uint64 * n)(), (C.c_uint64 * n)(), (C.c_int32 * n)()
+    rc = lib().palsgd_plan_layout(C.byref(cfg), n, nm, C.byref(bufs), C.byref(ns), C.byref(nc), C.byref(ce),
+                                  first, count, head)
+    if rc:
+        raise PalsgdError(rc, "palsgd_plan_layout")
+    return {"n_segments": ns.value, "n_chunks": nc.value, "chunk_elems": ce.value,
+            "segments": [(first[i], count[i], head[i]) for i in range(ns.value)]}
 
 
 class Palsgd:

@@ -305,15 +305,11 @@ int launch_inner(palsgd_ctx* ctx, const InnerArgs& a, cudaStream_t s)
     });
 }
 
-}  // namespace
-
-// ------------------------------------------------------------------------- init
-
-extern "C" int palsgd_init(palsgd_ctx** out, const palsgd_config* cfg, size_t n_tensors,
-                           const uint64_t* numel, const palsgd_buffers* bufs, void* stream)
+// Host-only planning of a tensor list: argument checks, fusion of adjacent tensors into segments, the
+// alignment head of every segment.  Looks at the ADDRESSES in `bufs` only, never at what they point to.
+int plan_segments(const palsgd_config* cfg, size_t n_tensors, const uint64_t* numel, const palsgd_buffers* bufs,
+                  std::vector<Segment>& segs, uint64_t& P)
 {
-    if (!out) return PALSGD_EINVAL;
-    *out = nullptr;
     int rc = validate_config(cfg);
     if (rc) return rc;
     if (n_tensors == 0 || !numel || !bufs) return PALSGD_EINVAL;
@@ -331,7 +327,7 @@ extern "C" int palsgd_init(palsgd_ctx** out, const palsgd_config* cfg, size_t n_
     struct Kind { int id; size_t esize; bool present; };
     const Kind kinds[5] = {{0, ps, true}, {1, ps, true}, {2, 4, bf}, {3, 4, true}, {4, 4, adam}};
 
-    uint64_t P = 0;
+    P = 0;
     for (size_t j = 0; j < n_tensors; ++j) {
         if (numel[j] > (1ull << 40)) return PALSGD_EINVAL;
         P += numel[j];
@@ -351,22 +347,6 @@ extern "C" int palsgd_init(palsgd_ctx** out, const palsgd_config* cfg, size_t n_
             if (!aligned(bufs->outer_v[j], 4)) return PALSGD_EALIGN;
         }
     }
-
-    palsgd_ctx* ctx = new (std::nothrow) palsgd_ctx();
-    if (!ctx) return PALSGD_ENOMEM;
-    ctx->cfg = *cfg;
-    ctx->n_tensors = n_tensors;
-    ctx->numel.assign(numel, numel + n_tensors);
-    ctx->P = P;
-    ctx->thr = threshold_of(cfg->p);
-    ctx->outer_lr = cfg->outer_lr;
-    // work item of the outer kernel, measured on B200: 1024 elements; for K = 5..7 (K + 2 streams per element,
-    // 4 CTAs per SM) larger items amortise the per-item prologue; K <= 4 runs the narrow-batch form of the
-    // kernel with 5 CTAs per SM, which does best with the small item (2048 for K <= 2)
-    ctx->outer_sub_elems = (K > 4 && K < 8) ? 4096u : K <= 2 ? 2048u : kOuterSubElems;
-    ctx->ddp_sub_elems = kDdpSubElems;
-    ctx->h_grad_dev.assign(bufs->grad, bufs->grad + (size_t)K * n_tensors);
-    ctx->h_global_dev.assign(bufs->global, bufs->global + n_tensors);
 
     // ---- fuse tensors that are adjacent in every buffer into segments
     auto adjacent = [&](size_t j) {           // is tensor j+1 right behind tensor j everywhere?
@@ -423,13 +403,56 @@ extern "C" int palsgd_init(palsgd_ctx** out, const palsgd_config* cfg, size_t n_
         j += sg.n_tensors;
         // (an empty tensor between two adjacent ones is skipped over by the fusion above; the first
         //  tensor of a non-empty segment may itself be empty, its pointer still marks the start)
-        if (sg.numel > 0) { sg.head = head_of(sg.first_tensor); ctx->segs.push_back(sg); }
+        if (sg.numel > 0) { sg.head = head_of(sg.first_tensor); segs.push_back(sg); }
     }
+    return PALSGD_OK;
+}
+
+// Elements per inner work item, measured best on B200: 4096 for fp32 AdamW, 8192 otherwise.
+inline uint32_t chunk_elems_for(const palsgd_config& cfg)
+{
+    return (cfg.precision != PALSGD_PREC_BF16_MASTER && cfg.inner == PALSGD_INNER_ADAMW) ? 4096u : kChunkElems;
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------------- init
+
+extern "C" int palsgd_init(palsgd_ctx** out, const palsgd_config* cfg, size_t n_tensors,
+                           const uint64_t* numel, const palsgd_buffers* bufs, void* stream)
+{
+    if (!out) return PALSGD_EINVAL;
+    *out = nullptr;
+    std::vector<Segment> planned;
+    uint64_t P = 0;
+    int rc = plan_segments(cfg, n_tensors, numel, bufs, planned, P);
+    if (rc) return rc;
+    const uint32_t K = cfg->K;
+    const bool bf = cfg->precision == PALSGD_PREC_BF16_MASTER;
+    const bool adam = cfg->inner == PALSGD_INNER_ADAMW;
+    const bool oadam = cfg->outer_opt == PALSGD_OUTER_ADAMW;
+
+    palsgd_ctx* ctx = new (std::nothrow) palsgd_ctx();
+    if (!ctx) return PALSGD_ENOMEM;
+    ctx->cfg = *cfg;
+    ctx->n_tensors = n_tensors;
+    ctx->numel.assign(numel, numel + n_tensors);
+    ctx->P = P;
+    ctx->thr = threshold_of(cfg->p);
+    ctx->outer_lr = cfg->outer_lr;
+    // work item of the outer kernel, measured on B200: 1024 elements; for K = 5..7 (K + 2 streams per element,
+    // 4 CTAs per SM) larger items amortise the per-item prologue; K <= 4 runs the narrow-batch form of the
+    // kernel with 5 CTAs per SM, which does best with the small item (2048 for K <= 2)
+    ctx->outer_sub_elems = (K > 4 && K < 8) ? 4096u : K <= 2 ? 2048u : kOuterSubElems;
+    ctx->ddp_sub_elems = kDdpSubElems;
+    ctx->h_grad_dev.assign(bufs->grad, bufs->grad + (size_t)K * n_tensors);
+    ctx->h_global_dev.assign(bufs->global, bufs->global + n_tensors);
+
+    ctx->segs = std::move(planned);
     const size_t n_seg = ctx->segs.size();
 
     // ---- chunk table of the inner kernel; item tables of the outer-sync and DDP kernels
-    // Elements per inner work item, measured best on B200: 4096 for fp32 AdamW, 8192 otherwise.
-    ctx->chunk_elems = (!bf && adam) ? 4096u : kChunkElems;
+    ctx->chunk_elems = chunk_elems_for(*cfg);
     const std::vector<Chunk> chunks = cut_segments(ctx->segs, ctx->chunk_elems);
     const std::vector<Chunk> oitems = cut_segments(ctx->segs, ctx->outer_sub_elems);
     const std::vector<Chunk> ditems = cut_segments(ctx->segs, ctx->ddp_sub_elems);
@@ -1078,6 +1101,27 @@ extern "C" int palsgd_get_launch_count(palsgd_ctx* ctx, uint64_t* n_launches)
 {
     if (!ctx || !n_launches) return PALSGD_EINVAL;
     *n_launches = ctx->launches;
+    return PALSGD_OK;
+}
+
+extern "C" int palsgd_plan_layout(const palsgd_config* cfg, size_t n_tensors, const uint64_t* numel,
+                                  const palsgd_buffers* bufs, uint64_t* n_segments, uint64_t* n_chunks,
+                                  uint32_t* chunk_elems, uint64_t* seg_first_tensor, uint64_t* seg_n_tensors,
+                                  int32_t* seg_head)
+{
+    std::vector<Segment> segs;
+    uint64_t P = 0;
+    const int rc = plan_segments(cfg, n_tensors, numel, bufs, segs, P);
+    if (rc) return rc;
+    const uint32_t ce = chunk_elems_for(*cfg);
+    if (n_segments) *n_segments = segs.size();
+    if (n_chunks) *n_chunks = cut_segments(segs, ce).size();
+    if (chunk_elems) *chunk_elems = ce;
+    for (size_t i = 0; i < segs.size(); ++i) {
+        if (seg_first_tensor) seg_first_tensor[i] = segs[i].first_tensor;
+        if (seg_n_tensors) seg_n_tensors[i] = segs[i].n_tensors;
+        if (seg_head) seg_head[i] = segs[i].head;
+    }
     return PALSGD_OK;
 }
 

@@ -5,6 +5,7 @@ import numpy as np
 import pytest
 import torch
 
+import paper_2504_18454_b200 as pkg
 import workloads as W
 from workloads.configs import WorkloadConfig
 from _harness import GpuRun, compare_state, make_oracle
@@ -312,6 +313,21 @@ def test_step_host_validates_the_result_pointers_before_anything_is_enqueued():
         assert np.array_equal(before[key], after[key]), key
     assert gpu.lib.step_host(gp, cfg.lr, cfg.eta, good, 0, gpu.stream) is True     # the context is still usable
     assert gpu.counters()["n_outer"] == 1
+
+
+@pytest.mark.parametrize("layout", ["arena", "separate", "misaligned"])
+@pytest.mark.parametrize("precision", [0, 1])
+def test_the_host_only_plan_agrees_with_what_init_built(layout, precision):
+    numel = [8192 * 2 + 5, 7, 0, 100, 300]
+    cfg = _cfg(numel, precision=precision)
+    gpu = GpuRun(cfg, _x0(cfg.K, sum(numel)), numel=numel, layout=layout, row_align=256)
+    addr = lambda name: [[int(t.data_ptr()) for t in row] for row in gpu.views[name]]
+    plan = pkg.plan_layout(K=cfg.K, numel=numel, precision=precision, inner=cfg.inner, param=addr("param"),
+                         grad=addr("grad"), m=addr("m"), v=addr("v"), master=addr("master") if precision else None,
+                         global_=addr("global_")[0], outer_mom=addr("outer_mom")[0])
+    built = gpu.lib.get_layout()
+    assert {k: plan[k] for k in built} == built
+    assert sum(n for _, n, _ in plan["segments"]) <= len(numel) and all(-1 <= h < 256 for _, _, h in plan["segments"])
 
 
 def test_layout_report_counts_segments_and_chunks():
