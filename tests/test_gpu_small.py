@@ -86,6 +86,33 @@ def test_long_scalar_head_in_front_of_a_list_one_element_off_a_256_element_grid(
     assert gpu.counters()["n_outer"] == orc.n_outer >= 2 and gpu.guards_intact()
 
 
+@pytest.mark.parametrize("layout,precision", [("separate", 0), ("separate", 1), ("arena", 1)])
+def test_thousands_of_small_tensors(layout, precision):
+    # one segment per tensor when every tensor is its own allocation: 3000 segments, most of them far smaller than
+    # a work item, some empty, a few spanning several chunks
+    rng = np.random.default_rng(17)
+    numel = [int(n) for n in rng.integers(0, 300, size=3000)]
+    for j in (5, 1500, 2999):
+        numel[j] = 8192 * 2 + 77
+    cfg = _cfg(numel, K=2, H=2, T=4, precision=precision)
+    gpu, orc, _ = _run_both(cfg, numel, layout, check_every_step=False)
+    lay = gpu.lib.get_layout()
+    nonempty = [n > 0 for n in numel]
+    runs = sum(1 for j, ne in enumerate(nonempty) if ne and (j == 0 or not nonempty[j - 1]))
+    # (packed: an empty tensor reports a NULL pointer, which ends a run of adjacent tensors)
+    if layout == "separate":     # (two allocations that happen to sit back to back in every buffer are fused: rare)
+        assert 0.98 * sum(nonempty) <= lay["n_segments"] <= sum(nonempty)
+    else:
+        assert lay["n_segments"] == runs
+    gpu.set_grad_clip(0.01); orc.set_grad_clip(0.01)
+    P_ = int(sum(numel))
+    for t in range(4, 6):
+        g = _grads(cfg, P_, t)
+        gpu.set_grads(g); gpu.step(cfg.lr, cfg.eta); orc.step(g, cfg.lr, cfg.eta)
+    compare_state(gpu.state(), orc, exact=True)
+    assert gpu.guards_intact()
+
+
 @pytest.mark.parametrize("K", [1, 2, 3, 8, 32, 64])
 def test_worker_counts(K):
     numel = [4096 * 2 + 13]
