@@ -137,6 +137,18 @@ def test_extreme_probabilities(p):
         assert c["s"] == [0] * 4             # always pulls
 
 
+@pytest.mark.parametrize("precision", [0, 1])
+def test_zero_step_size_and_zero_mixing_rate(precision):
+    numel = [5000]
+    # eta = 0: the pull coefficient is 0, a pulling worker keeps its model (and takes no gradient step)
+    gpu, orc, _ = _run_both(_cfg(numel, eta=0.0, p=0.5, H=4, T=8, precision=precision), numel, "arena")
+    # alpha = 0: the gradient branch moves the moments only
+    x0 = _x0(4, 5000, same=True)
+    gpu, orc, _ = _run_both(_cfg(numel, lr=0.0, p=0.5, H=4, T=3, precision=precision), numel, "arena", x0=x0)
+    st = gpu.state()
+    assert np.array_equal(st["x"], x0) and np.any(st["m"] != 0)
+
+
 def test_plain_averaging_outer_and_momentum_without_nesterov():
     numel = [9000]
     _run_both(_cfg(numel, outer_lr=1.0, outer_momentum=0.0, outer_nesterov=False, H=3, T=6), numel, "arena")
