@@ -282,6 +282,134 @@ def workload_config(cfg, args) -> dict:
 
 # ----------------------------------------------------------------------------- GPU leg
 
+def run_workers(args, cfg):
+    """The deployment the paper runs: the K workers spread over the ranks (K / world each, one rank per GPU),
+    inner steps local, every H steps the outer sync as local sum -> all-reduce(sum) over NCCL -> finish
+    (Algorithm 1's All-Reduce).  Total work is fixed as the ranks grow ("strong").  One JSON line from rank 0."""
+    import torch
+    import torch.distributed as dist
+    import paper_2504_18454_b200 as P
+    from paper_2504_18454_b200.arena import ReplicaArena
+    from paper_2504_18454_b200.workers import DistributedPalsgd, worker_span
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.gpus > 1 and world != args.gpus:
+        raise SystemExit("launch with: python -m torch.distributed.run --nnodes=1 --nproc-per-node N "
+                         "--master-addr 127.0.0.1 --master-port P bench.py --gpus N --workers ...")
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if "RANK" in os.environ:                             # under torchrun, one rank included: the collective is NCCL's
+        dist.init_process_group("nccl", device_id=dev)
+    k0, k1 = worker_span(cfg.K, rank, world)
+    K, Kl, Pn = cfg.K, k1 - k0, cfg.P
+    numel = [t.numel for t in cfg.tensors]
+
+    def barrier():
+        if dist.is_initialized():
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    arena = ReplicaArena(numel, Kl, precision=cfg.precision, inner=cfg.inner, device=dev)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(cfg.param_seed)                      # one initial model for the whole job (Algorithm 1)
+    x0 = torch.randn(Pn, generator=gen, device=dev).mul_(cfg.init_std)
+    for k in range(Kl):
+        arena.write_flat(arena.model_name, k, x0)
+        gen.manual_seed(cfg.grad_seed + k0 + k)          # one gradient per worker of the job
+        arena.write_flat("grad", k, torch.randn(Pn, generator=gen, device=dev).mul_(cfg.grad_std))
+    del x0
+    stream = torch.cuda.current_stream(dev).cuda_stream
+    ctx = arena.make_context(
+        stream=stream, H=cfg.H, p=cfg.p, beta1=cfg.beta1, beta2=cfg.beta2, eps=cfg.eps, weight_decay=cfg.weight_decay,
+        momentum=cfg.momentum, outer_lr=cfg.outer_lr, outer_momentum=cfg.outer_momentum,
+        outer_nesterov=cfg.outer_nesterov, seed=cfg.decision_seed)
+    exch = torch.zeros(ctx.exchange_numel(), dtype=torch.float32, device=dev)
+
+    def all_reduce_sum(buf):
+        if dist.is_initialized():
+            dist.all_reduce(buf, op=dist.ReduceOp.SUM)   # on torch's current stream, the one the kernels use
+
+    job = DistributedPalsgd(ctx, exch, K, rank, world, all_reduce_sum=all_reduce_sum)
+    job.init_global(stream)
+
+    def one_step(rec=None):
+        ev = lambda: torch.cuda.Event(enable_timing=True)
+        e = [ev() for _ in range(5)]
+        e[0].record(); ctx.inner_step(cfg.lr, cfg.eta, stream); job.t += 1; e[1].record()
+        if job.t % cfg.H == 0:
+            ctx.outer_partial(exch.data_ptr(), stream); e[2].record()
+            all_reduce_sum(exch); e[3].record()
+            ctx.outer_finish(exch.data_ptr(), K, stream); e[4].record()
+            if rec is not None:
+                rec.append(("sync", job.t, e))
+        elif rec is not None:
+            rec.append(("inner", job.t, e))
+
+    for _ in range(max(args.warmup, 3)):
+        one_step()
+    while job.t % cfg.H != 0:                            # the timed region starts right behind a synchronisation
+        one_step()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    launches0 = ctx.get_launch_count()
+    rec = []
+    barrier()
+    e_start = torch.cuda.Event(enable_timing=True); e_end = torch.cuda.Event(enable_timing=True)
+    e_start.record()
+    for _ in range(args.steps):
+        one_step(rec)
+    e_end.record()
+    barrier()
+    ms_total = e_start.elapsed_time(e_end)
+    launches = ctx.get_launch_count() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+
+    inner_ms = inner_bytes = part_ms = coll_ms = fin_ms = 0.0
+    n_sync = 0
+    for kind, t_after, e in rec:
+        inner_ms += e[0].elapsed_time(e[1])
+        inner_bytes += sum(inner_bytes_per_element(cfg, bool(P.decision(cfg.decision_seed, t_after - 1, k0 + k, cfg.p)))
+                           for k in range(Kl)) * Pn
+        if kind == "sync":
+            part_ms += e[1].elapsed_time(e[2]); coll_ms += e[2].elapsed_time(e[3]); fin_ms += e[3].elapsed_time(e[4])
+            n_sync += 1
+    ms_total, inner_ms, part_ms, coll_ms, fin_ms = max_over_ranks([ms_total, inner_ms, part_ms, coll_ms, fin_ms], world, dev)
+    if dist.is_initialized():
+        dist.destroy_process_group()
+    if rank != 0:
+        return
+    peak, peak_src = measured_peak_gbs()
+    g_es = 2 if cfg.precision == 1 else 4
+    sync_part = lambda name, ms, per_param: ({"kernel": name, "avg_ms": ms / n_sync,
+                                              "achieved": per_param * Pn * n_sync / (ms * 1e-3) / 1e9, "unit": "GB/s"}
+                                             if n_sync and ms > 0 else None)
+    out = {
+        "metric": METRIC, "value": K * Pn * args.steps / (ms_total * 1e-3), "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_total / args.steps,
+        "higher_is_better": True, "scaling": "strong", "vs_baseline": None, "dtype": dtype_of(cfg), "data": "synthetic",
+        "config": dict(workload_config(cfg, args), parallelism=f"{Kl} of the {K} workers per GPU; outer sync as local "
+                       f"sum -> all-reduce(sum) of {Pn} floats -> finish every H steps"),
+        "roofline": roofline_entry("palsgd_inner_kernel", "inner", cfg, peak, peak_src, inner_ms, inner_bytes, len(rec),
+                                   units_per_launch=Kl * Pn, traffic=None),
+        "outer_exchange": {"syncs": n_sync,
+                           "partial": sync_part("palsgd_outer_partial_kernel", part_ms, 4 * Kl + 4),
+                           "all_reduce": ({"avg_ms": coll_ms / n_sync, "bytes": 4 * Pn,
+                                           "backend": "nccl" if world > 1 or "RANK" in os.environ else "none (one rank)"}
+                                          if n_sync else None),
+                           "finish": sync_part("palsgd_outer_kernel (sum from the exchange buffer)", fin_ms,
+                                               (6 if cfg.precision == 1 else 4) * Kl + 20)},
+        "cpu_baseline": None, "e2e": None, "gpu_launches": launches, "clocks": clocks,
+        "note": "workers spread over the ranks; times are the maximum over ranks; gradients stay resident (no end-to-end "
+                "leg in this mode)",
+    }
+    print(json.dumps(out), flush=True)
+
+
 def run_ours(args, cfg):
     import torch
     import torch.distributed as dist
@@ -644,6 +772,9 @@ def main():
     ap.add_argument("--shard", action="store_true",
                     help="N > 1: one model sharded over the ranks along the parameter axis (strong scaling, no "
                          "exchange) instead of one replica of the workload per rank")
+    ap.add_argument("--workers", action="store_true",
+                    help="spread the K workers over the ranks (K / N each) and run the outer sync around an NCCL "
+                         "all-reduce: the paper's own deployment; not the default")
     ap.add_argument("--layout", choices=["arena", "separate", "misaligned"], default="arena",
                     help="device layout of the tensor list: packed (K, P) arenas (default), one allocation per "
                          "(worker, tensor, buffer kind), or packed and shifted off 16-byte alignment")
@@ -662,6 +793,8 @@ def main():
         if args.steps == 256:
             args.steps = 32                       # a bounded sample: keep the CPU run to about a minute
         run_reference(args, cfg)
+    elif args.workers:
+        run_workers(args, cfg)
     else:
         run_ours(args, cfg)
 

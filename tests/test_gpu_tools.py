@@ -71,3 +71,20 @@ def test_default_layout_run_also_times_the_ragged_layout():
     assert rg["roofline"]["launches"] == 16 and rg["roofline"]["achieved"] > 0 and rg["roofline"]["traffic"] is None
     assert rg["roofline_outer"]["launches"] == 4 and rg["roofline_outer"]["achieved"] > 0
     assert d["gpu_launches"] == 4                      # the extra region is not part of the timed step loop
+
+
+@pytest.mark.parametrize("launcher", ["plain", "torchrun"])
+def test_bench_workers_mode_runs_with_one_rank(launcher):
+    # the paper's deployment (workers spread over the ranks, outer sync around an all-reduce) with the one rank a
+    # single GPU allows: plain (no process group) and under torchrun (NCCL process group of one rank)
+    tail = ["bench.py", "--gpus", "1", "--workers", "--workload", "c0_flat_1m", "--steps", "16", "--warmup", "3"]
+    head = [] if launcher == "plain" else ["-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", "1",
+                                           "--master-addr", "127.0.0.1", "--master-port", "29643"]
+    out = _run(head + tail)
+    d = json.loads([l for l in out.splitlines() if l.startswith("{")][-1])
+    assert d["scaling"] == "strong" and d["n_gpus"] == 1 and d["value"] > 0
+    ex = d["outer_exchange"]
+    assert ex["syncs"] == 2 and ex["partial"]["achieved"] > 0 and ex["finish"]["achieved"] > 0     # H = 8
+    assert ex["all_reduce"]["bytes"] == 4 * (1 << 20)
+    assert ex["all_reduce"]["backend"] == ("nccl" if launcher == "torchrun" else "none (one rank)")
+    assert d["roofline"]["achieved"] > 0 and d["gpu_launches"] == 16 + 2 * 2
