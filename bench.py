@@ -339,7 +339,7 @@ def run_workers(args, cfg):
     def one_step(rec=None):
         ev = lambda: torch.cuda.Event(enable_timing=True)
         e = [ev() for _ in range(5)]
-        e[0].record(); ctx.inner_step(cfg.lr, cfg.eta, stream); job.t += 1; e[1].record()
+        e[0].record(); job.inner_step(cfg.lr, cfg.eta, stream); e[1].record()       # (counts the step in job.t)
         if job.t % cfg.H == 0:
             ctx.outer_partial(exch.data_ptr(), stream); e[2].record()
             all_reduce_sum(exch); e[3].record()
