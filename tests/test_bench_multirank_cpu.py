@@ -26,7 +26,9 @@ dist.destroy_process_group()
 '''
 
 
-def _torchrun(args, port):
+def _torchrun(args, port=None):
+    from conftest import free_port
+    port = free_port()                  # whatever the caller asked for: a port that is free now
     env = dict(os.environ, MASTER_ADDR="127.0.0.1", OMP_NUM_THREADS="1")
     cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", "2",
            "--master-addr", "127.0.0.1", "--master-port", str(port)] + args

@@ -75,11 +75,12 @@ def test_default_layout_run_also_times_the_ragged_layout():
 
 @pytest.mark.parametrize("launcher", ["plain", "torchrun"])
 def test_bench_workers_mode_runs_with_one_rank(launcher):
+    from conftest import free_port
     # the paper's deployment (workers spread over the ranks, outer sync around an all-reduce) with the one rank a
     # single GPU allows: plain (no process group) and under torchrun (NCCL process group of one rank)
     tail = ["bench.py", "--gpus", "1", "--workers", "--workload", "c0_flat_1m", "--steps", "16", "--warmup", "3"]
     head = [] if launcher == "plain" else ["-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", "1",
-                                           "--master-addr", "127.0.0.1", "--master-port", "29643"]
+                                           "--master-addr", "127.0.0.1", "--master-port", str(free_port())]
     out = _run(head + tail)
     d = json.loads([l for l in out.splitlines() if l.startswith("{")][-1])
     assert d["scaling"] == "strong" and d["n_gpus"] == 1 and d["value"] > 0

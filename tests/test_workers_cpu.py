@@ -142,11 +142,12 @@ dist.destroy_process_group()
 
 
 def test_two_ranks_hold_half_of_the_workers_each(tmp_path):
+    from conftest import free_port
     script = tmp_path / "worker.py"
     script.write_text(WORKER)
     env = dict(os.environ, MASTER_ADDR="127.0.0.1", OMP_NUM_THREADS="1")
     cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", "2",
-           "--master-addr", "127.0.0.1", "--master-port", "29621", str(script), ROOT, str(tmp_path)]
+           "--master-addr", "127.0.0.1", "--master-port", str(free_port()), str(script), ROOT, str(tmp_path)]
     r = subprocess.run(cmd, cwd=ROOT, env=env, capture_output=True, text=True, timeout=600)
     assert r.returncode == 0, r.stderr[-3000:]
     for rank in (0, 1):
