@@ -305,6 +305,10 @@ int palsgd_cycle_launch(palsgd_ctx* ctx, void* stream);
  * the library's own (ordered after the work already enqueued on `stream`), and the part
  * of the inner step that belongs to worker k is launched when its gradient has arrived
  * (K launches per step; with gradient clipping on, or K = 1, one launch after all copies).
+ * A worker's SMALL copies (under 2 MB each, both ends 16-byte aligned, at least 8 of them, the
+ * sources in pinned memory -- a tensor list held as one allocation per tensor) are performed by
+ * one more kernel that reads the host memory directly, instead of one copy-engine transfer each;
+ * pageable sources and everything else go through cudaMemcpyAsync.  The data moved is the same.
  * Errors: as palsgd_step; EINVAL for a NULL gradient pointer of a non-empty tensor of a
  * worker that takes a gradient step, and for a NULL entry of h_global (non-empty tensor) on a
  * step that ends with the outer sync -- both found before anything is enqueued.

@@ -30,6 +30,38 @@ constexpr size_t kTwoStageLimit = 32 * 1024;
 constexpr int kOuterCtasPerSm = 0;
 constexpr int kDdpCtasPerSm = 4;
 
+// palsgd_step_host: one small host -> device copy that a kernel performs (see palsgd_gather_host_kernel).
+struct HostCopy {
+    const unsigned char* src;     // pinned host memory, through its device alias; 16-byte aligned
+    unsigned char*       dst;     // device memory, 16-byte aligned
+    uint64_t             bytes;
+};
+// Copies below this size go through the gather kernel when a worker has at least kGatherMinCopies of them.
+constexpr size_t kGatherMaxBytes = 2 * 1024 * 1024;    // measured: 256 KB, 1 MB and 16 MB all do worse on the three model-shaped lists
+constexpr size_t kGatherMinCopies = 8;
+constexpr size_t kGatherItemBytes = 32 * 1024;               // longer copies are cut into table entries of this size
+
+// The many small tensors of a framework-style layout (biases, normalisation scales: a few KB each) cost a copy
+// engine several microseconds apiece, whatever their size.  This kernel performs all of a worker's small copies
+// in one launch: every CTA takes whole entries of the table and reads the PINNED host memory directly (the
+// table itself lives there too).  Large tensors still travel through the copy engine.
+__global__ void __launch_bounds__(256) palsgd_gather_host_kernel(const HostCopy* __restrict__ items, uint32_t n_items)
+{
+    for (uint32_t it = blockIdx.x; it < n_items; it += gridDim.x) {
+        const HostCopy c = items[it];
+        const uint32_t n16 = (uint32_t)(c.bytes >> 4);       // (an entry is at most kGatherItemBytes long)
+        const uint4* __restrict__ s = reinterpret_cast<const uint4*>(c.src);
+        uint4* __restrict__ d = reinterpret_cast<uint4*>(c.dst);
+        uint32_t i = threadIdx.x;
+        for (; i + 3 * 256 < n16; i += 4 * 256) {            // four reads of host memory in flight per thread
+            const uint4 a0 = s[i], a1 = s[i + 256], a2 = s[i + 512], a3 = s[i + 768];
+            d[i] = a0; d[i + 256] = a1; d[i + 512] = a2; d[i + 768] = a3;
+        }
+        for (; i < n16; i += 256) d[i] = s[i];
+        for (uint32_t j = (n16 << 4) + threadIdx.x; j < c.bytes; j += 256) c.dst[j] = c.src[j];
+    }
+}
+
 struct Segment {
     size_t   first_tensor;
     size_t   n_tensors;
@@ -73,6 +105,8 @@ struct palsgd_ctx {
     cudaStream_t copy_stream = nullptr;           // palsgd_step_host: host -> device copies run here ...
     std::vector<cudaEvent_t> copy_done;           // ... and signal worker k's gradient with copy_done[k]
     cudaEvent_t copy_may_start = nullptr;         // recorded on the caller's stream before the copies begin
+    HostCopy* gather_items = nullptr;             // pinned host table of the small copies of one palsgd_step_host call
+    size_t gather_cap = 0;                        //   (read by palsgd_gather_host_kernel straight from host memory)
     cudaGraphExec_t cycle_exec = nullptr;         // captured H-step cycle (palsgd_cycle_capture) or nullptr
     uint64_t cycle_launches = 0;                  // kernels inside one captured cycle
     int sm_count = 0, smem_optin = 0;             // device attributes read at init
@@ -919,8 +953,14 @@ extern "C" int palsgd_step_host(palsgd_ctx* ctx, const void* const* h_grad, doub
     // host -> device gradients of worker k; tensors adjacent on both sides travel as one copy.
     // A worker that pulls in this step has no use for a gradient (Algorithm 1 takes one branch or the
     // other), so nothing is transferred for it.
+    // Small copies (under kGatherMaxBytes, both ends 16-byte aligned, the source pinned) are collected and, if a
+    // worker has kGatherMinCopies or more of them, performed by one launch of the gather kernel on the same stream.
+    std::vector<HostCopy> small, pieces;
+    std::vector<const unsigned char*> alias;
+    size_t gather_used = 0;                                  // entries of the pinned table taken by earlier workers
     auto copy_worker = [&](uint32_t k, cudaStream_t cs) -> int {
         if (draw_pull(ctx->cfg.seed, ctx->t, ctx->k0 + k, ctx->thr)) return PALSGD_OK;
+        small.clear();
         for (const Segment& sg : ctx->segs) {
             size_t j = sg.first_tensor;
             const size_t end = sg.first_tensor + sg.n_tensors;
@@ -933,12 +973,68 @@ extern "C" int palsgd_step_host(palsgd_ctx* ctx, const void* const* h_grad, doub
                     bytes += ctx->numel[j2] * gs;
                     ++j2;
                 }
-                if (bytes)
-                    PALSGD_CUDA(ctx, cudaMemcpyAsync(const_cast<void*>(ctx->h_grad_dev[idx]), src, bytes,
-                                                     cudaMemcpyHostToDevice, cs));
+                void* dst = const_cast<void*>(ctx->h_grad_dev[idx]);
+                if (bytes && bytes < kGatherMaxBytes && aligned(src, 16) && aligned(dst, 16)) {
+                    small.push_back(HostCopy{reinterpret_cast<const unsigned char*>(src),
+                                             static_cast<unsigned char*>(dst), bytes});
+                } else if (bytes)
+                    PALSGD_CUDA(ctx, cudaMemcpyAsync(dst, src, bytes, cudaMemcpyHostToDevice, cs));
                 j = j2;
             }
         }
+        // the kernel may only read memory the device can reach: every source is looked up (pinned or not, and
+        // its device alias) on every call -- a buffer may have been replaced since the last one
+        bool gather = small.size() >= kGatherMinCopies;
+        alias.assign(small.size(), nullptr);                 // the sources as the device addresses them
+        for (size_t i = 0; gather && i < small.size(); ++i) {
+            cudaPointerAttributes at{};
+            if (cudaPointerGetAttributes(&at, small[i].src) != cudaSuccess) { (void)cudaGetLastError(); gather = false; break; }
+            if (at.type != cudaMemoryTypeHost || !at.devicePointer) { gather = false; break; }
+            // the whole range must lie inside the same registration: the last byte is looked up as well
+            cudaPointerAttributes at_end{};
+            if (cudaPointerGetAttributes(&at_end, small[i].src + small[i].bytes - 1) != cudaSuccess ||
+                at_end.type != cudaMemoryTypeHost) { (void)cudaGetLastError(); gather = false; break; }
+            alias[i] = static_cast<const unsigned char*>(at.devicePointer);
+        }
+        if (gather) {                                        // cut into table entries of at most kGatherItemBytes
+            pieces.clear();
+            for (size_t i = 0; i < small.size(); ++i)
+                for (uint64_t off = 0; off < small[i].bytes; off += kGatherItemBytes)
+                    pieces.push_back(HostCopy{alias[i] + off, small[i].dst + off,
+                                              std::min<uint64_t>(kGatherItemBytes, small[i].bytes - off)});
+        }
+        if (gather) {
+            const size_t need = gather_used + pieces.size();
+            if (need > ctx->gather_cap) {
+                // grow the pinned table; earlier workers' launches of this call still read the old one
+                if (gather_used > 0) PALSGD_CUDA(ctx, cudaStreamSynchronize(cs));
+                HostCopy* bigger = nullptr;
+                const size_t cap = std::max(need, (size_t)K * pieces.size()) + 64;
+                if (cudaHostAlloc(reinterpret_cast<void**>(&bigger), cap * sizeof(HostCopy), cudaHostAllocDefault) != cudaSuccess) {
+                    (void)cudaGetLastError();
+                    gather = false;                          // no table: the copy engine takes them
+                } else {
+                    if (ctx->gather_items) cudaFreeHost(ctx->gather_items);
+                    ctx->gather_items = bigger;
+                    ctx->gather_cap = cap;
+                    gather_used = 0;
+                }
+            }
+        }
+        if (gather) {
+            HostCopy* table = ctx->gather_items + gather_used;
+            std::memcpy(table, pieces.data(), pieces.size() * sizeof(HostCopy));
+            gather_used += pieces.size();
+            void* table_dev = nullptr;
+            PALSGD_CUDA(ctx, cudaHostGetDevicePointer(&table_dev, table, 0));
+            const uint32_t n_items = (uint32_t)pieces.size();
+            const unsigned grid = grid_for(n_items, ctx->sm_count > 0 ? ctx->sm_count * 8 : 1184);
+            return launch_checked(ctx, [&] {
+                palsgd_gather_host_kernel<<<grid, 256, 0, cs>>>(static_cast<const HostCopy*>(table_dev), n_items);
+            });
+        }
+        for (const HostCopy& c : small)
+            PALSGD_CUDA(ctx, cudaMemcpyAsync(c.dst, c.src, c.bytes, cudaMemcpyHostToDevice, cs));
         return PALSGD_OK;
     };
     InnerArgs a = inner_args(ctx, lr_t, eta_t);
@@ -1207,6 +1303,7 @@ extern "C" void palsgd_destroy(palsgd_ctx* ctx)
     for (cudaEvent_t e : ctx->copy_done) if (e) cudaEventDestroy(e);
     if (ctx->copy_may_start) cudaEventDestroy(ctx->copy_may_start);
     if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
+    if (ctx->gather_items) cudaFreeHost(ctx->gather_items);
     if (ctx->d_oitems) cudaFree(ctx->d_oitems);
     if (ctx->d_ditems) cudaFree(ctx->d_ditems);
     if (ctx->d_blob) cudaFree(ctx->d_blob);

@@ -326,6 +326,46 @@ def test_step_host_transfers_no_gradient_for_workers_that_pull_and_splits_the_st
     assert gpu.counters()["s"] == [int(v) for v in orc.s]
 
 
+@pytest.mark.parametrize("pinned", [True, False])
+@pytest.mark.parametrize("precision", [0, 1])
+def test_step_host_with_many_small_tensors_gathers_them_in_one_launch_per_worker(pinned, precision):
+    # one allocation per tensor on the device, 60 small tensors: from pinned memory a worker's small copies are
+    # performed by one launch of the gather kernel (plus the copy engine for the large tensor and for sources off
+    # 16-byte alignment); from pageable memory everything goes through the copy engine.  Same results either way.
+    rng = np.random.default_rng(3)
+    numel = [int(n) for n in rng.choice([8, 64, 256, 768, 1000, 3072], size=60)] + [7, 300000, 0, 5, 128]
+    P = sum(numel)
+    cfg = _cfg(numel, K=3, p=0.3, H=2, precision=precision)
+    x0 = _x0(cfg.K, P, same=True)
+    gpu, orc = GpuRun(cfg, x0, numel=numel, layout="separate"), make_oracle(cfg, x0)
+    gdt = torch.bfloat16 if precision else torch.float32
+    hg = torch.empty((cfg.K, P), dtype=gdt)
+    hg = hg.pin_memory() if pinned else hg
+    es = hg.element_size()
+    starts = np.concatenate([[0], np.cumsum(numel)])
+    gp = gpu.lib.make_ptr_array([hg.data_ptr() + (k * P + int(starts[j])) * es
+                                 for k in range(cfg.K) for j in range(len(numel))])
+    import paper_2504_18454_b200 as PL
+    launches, expected = gpu.lib.get_launch_count(), 0
+    for t in range(4):
+        g = _grads(cfg, P, t)
+        src = torch.from_numpy(g.view(np.int16)).view(torch.bfloat16) if precision else torch.from_numpy(g)
+        hg.copy_(src)
+        gpu.lib.step_host(gp, cfg.lr, cfg.eta, None, 0, gpu.stream)
+        orc.step(g, cfg.lr, cfg.eta)
+        takes_gradient = [1 - PL.decision(cfg.decision_seed, t, k, cfg.p) for k in range(cfg.K)]
+        expected += cfg.K + (sum(takes_gradient) if pinned else 0) + (1 if (t + 1) % cfg.H == 0 else 0)
+        on_device = gpu._read("grad")
+        for k in range(cfg.K):
+            if takes_gradient[k]:
+                assert np.array_equal(on_device[k], g[k]), (t, k)
+    compare_state(gpu.state(), orc, exact=True)
+    # (a worker whose small copies are mostly off 16-byte alignment on the host keeps to the copy engine)
+    got, plain = gpu.lib.get_launch_count() - launches, 4 * cfg.K + 2
+    assert plain < got <= expected if pinned else got == expected == plain
+    assert gpu.guards_intact()
+
+
 def test_step_host_validates_the_result_pointers_before_anything_is_enqueued():
     # a NULL entry in h_global on a step that ends with an outer sync: EINVAL, and nothing has moved
     numel = [3000, 40]
