@@ -366,6 +366,33 @@ def test_step_host_with_many_small_tensors_gathers_them_in_one_launch_per_worker
     assert gpu.guards_intact()
 
 
+def test_step_host_gather_table_grows_inside_one_call():
+    # worker 0's host row has 10 small tensors on 16-byte boundaries and 300 off them, worker 1's row the other way
+    # round, so the pinned table sized after worker 0 is too small for worker 1 and has to grow in mid-call
+    numel = [16] * 10 + [1] + [16] * 300
+    P = sum(numel)
+    cfg = _cfg(numel, K=3, p=0.0, H=2, inner=1, momentum=0.9)
+    x0 = _x0(cfg.K, P, same=True)
+    gpu, orc = GpuRun(cfg, x0, numel=numel, layout="separate"), make_oracle(cfg, x0)
+    pitch, shift = (P + 8 + 3) // 4 * 4, [0, 3, 0]                              # elements; worker 1's row starts 12 bytes late
+    hg = torch.empty(cfg.K * pitch, dtype=torch.float32).pin_memory()
+    assert hg.data_ptr() % 16 == 0 and pitch % 4 == 0
+    rows = [hg[k * pitch + shift[k]: k * pitch + shift[k] + P] for k in range(cfg.K)]
+    starts = np.concatenate([[0], np.cumsum(numel)])
+    gp = gpu.lib.make_ptr_array([rows[k].data_ptr() + int(starts[j]) * 4 for k in range(cfg.K) for j in range(len(numel))])
+    launches = gpu.lib.get_launch_count()
+    for t in range(3):
+        g = _grads(cfg, P, t)
+        for k in range(cfg.K):
+            rows[k].copy_(torch.from_numpy(g[k]))
+        gpu.lib.step_host(gp, cfg.lr, cfg.eta, None, 0, gpu.stream)
+        orc.step(g, cfg.lr, cfg.eta)
+        assert np.array_equal(gpu._read("grad"), g)
+    compare_state(gpu.state(), orc, exact=True)
+    assert gpu.lib.get_launch_count() - launches == 3 * (cfg.K + cfg.K) + 1      # inner + gather per worker; one sync
+    assert gpu.guards_intact()
+
+
 def test_step_host_validates_the_result_pointers_before_anything_is_enqueued():
     # a NULL entry in h_global on a step that ends with an outer sync: EINVAL, and nothing has moved
     numel = [3000, 40]
